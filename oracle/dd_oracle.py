@@ -1,0 +1,240 @@
+"""Plain CPU oracle of the per-layer sparse decode hot path (DualDecoder).
+
+TEST INFRASTRUCTURE ONLY: imported by tests, the smoke check and the CPU legs
+of the benchmark; never by the product package, and it never calls the CUDA
+library. Slow on purpose: every function is the definition written out in
+numpy, in fp64 unless a storage rounding is part of the definition.
+
+The paper defines the path in prose only (no equation, no listing):
+
+* retrieval index = f(token query, static GPU-resident chunk landmarks)
+  (Sec. 2.2 "Dynamic Sparse KV Cache", Sec. 4.1 "KV Retrieval Predictability");
+* the index used for step i+1 is predicted from the speculated token of step i
+  (Sec. 4.1 "Retrieval index prediction");
+* selected KV blocks are moved from host memory into a layer-scoped GPU buffer
+  in attention layout (Sec. 5.3, Sec. 5.4 "GPU-side sparse KV assembly");
+* attention runs over exactly that sparse set (Sec. 4.2, Sec. 5.4).
+
+Readings taken where the paper is silent (each is listed in the design notes):
+landmark = per-page mean key, stored in bf16; score = scaled dot product,
+softmax over the request's valid pages per query head, then maximum over the
+query heads that share a KV head; ties go to the lower page; the selected set
+is emitted in ascending page order; the last `forced_recent` valid pages are
+always selected and count inside the budget.
+
+Parity with numbers printed in the paper: UNPINNED for every function (the
+paper prints no worked example). Correctness is pinned by closed forms, brute
+force, invariants and library special cases in tests/test_oracle_*.py.
+
+Array conventions (numpy):
+  q        [B, Tq, Hq, d]   queries, token 0 = current, token 1 = speculated
+  lm       [B, Hkv, P, d]   landmarks (bf16-representable values)
+  kv       [B, Hkv, P, 2, T, d]  one layer of the host store, [..,0,..]=K, [..,1,..]=V
+  idx      [B, Hkv, k]      selected pages, ascending
+  slot     [B, Hkv, 2, k*T, d]   gathered buffer in attention layout
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "round_to_bf16",
+    "build_landmarks",
+    "page_scores",
+    "topk_pages",
+    "select_topk",
+    "gather_kv",
+    "sparse_decode_attn",
+    "decode_chain",
+]
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even); returns fp32.
+
+    bf16 is the upper 16 bits of an IEEE fp32, so rounding adds half of the
+    dropped field (plus the parity of the kept LSB) and truncates.
+    NaN is not expected on this path.
+    """
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    bits = a.view(np.uint32).astype(np.uint64)
+    lsb = (bits >> np.uint64(16)) & np.uint64(1)
+    bits = (bits + np.uint64(0x7FFF) + lsb) & np.uint64(0xFFFF0000)
+    return bits.astype(np.uint32).view(np.float32).reshape(a.shape)
+
+
+def build_landmarks(k_pages: np.ndarray, ctx_len: np.ndarray) -> np.ndarray:
+    """Landmark of a page = mean of its valid keys (Sec. 2.2: chunks of adjacent
+    KV entries with compressed landmarks; Sec. 4.1: built before decoding, fixed).
+
+    k_pages [B, Hkv, P, T, d] bf16-valued; ctx_len [B] tokens. A page with no
+    valid token gets a zero landmark (it is never scored). The storage format is
+    part of the definition: sum in fp32 in token order, divide in fp32, round to
+    bf16, so that the same bits can be produced by any implementation.
+    """
+    k_pages = np.asarray(k_pages, dtype=np.float32)
+    B, Hkv, P, T, d = k_pages.shape
+    out = np.zeros((B, Hkv, P, d), dtype=np.float32)
+    for b in range(B):
+        n_tok = int(ctx_len[b])
+        for p in range(P):
+            cnt = min(T, n_tok - p * T)
+            if cnt <= 0:
+                continue
+            acc = np.zeros((Hkv, d), dtype=np.float32)
+            for i in range(cnt):
+                acc = acc + k_pages[b, :, p, i, :]
+            out[b, :, p, :] = acc / np.float32(cnt)
+    return round_to_bf16(out)
+
+
+def page_scores(q_tok: np.ndarray, lm: np.ndarray, n_pages: int, group_reduce: str = "softmax_max"):
+    """Scores of one request's pages for every KV head (Sec. 4.1).
+
+    q_tok [Hq, d] (the scoring token's per-head queries), lm [Hkv, P, d].
+    Returns (score [Hkv, n_pages] in (0, 1], logit s [Hq, n_pages], lse [Hq]).
+
+      s[h, p]  = <q[h], lm[g(h), p]> / sqrt(d),  g(h) = h // (Hq / Hkv)
+      lse[h]   = log sum_p exp(s[h, p])          over the valid pages
+      score[g, p] = max_{h in group g} exp(s[h, p] - lse[h])
+
+    `group_reduce` other than "softmax_max" exists only to show sensitivity to
+    the reading ("logit_max", "logit_mean"); the contract is "softmax_max".
+    """
+    q_tok = np.asarray(q_tok, dtype=np.float64)
+    lm = np.asarray(lm, dtype=np.float64)
+    Hq, d = q_tok.shape
+    Hkv = lm.shape[0]
+    assert Hq % Hkv == 0
+    G = Hq // Hkv
+    s = np.empty((Hq, n_pages), dtype=np.float64)
+    for h in range(Hq):
+        s[h] = lm[h // G, :n_pages, :] @ q_tok[h] / np.sqrt(float(d))
+    m = s.max(axis=1, keepdims=True)
+    lse = (m + np.log(np.exp(s - m).sum(axis=1, keepdims=True)))[:, 0]
+    if group_reduce == "softmax_max":
+        per_head = np.exp(s - lse[:, None])
+        score = per_head.reshape(Hkv, G, n_pages).max(axis=1)
+    elif group_reduce == "logit_max":
+        score = s.reshape(Hkv, G, n_pages).max(axis=1)
+    elif group_reduce == "logit_mean":
+        score = s.reshape(Hkv, G, n_pages).mean(axis=1)
+    else:
+        raise ValueError(group_reduce)
+    return score, s, lse
+
+
+def topk_pages(score: np.ndarray, k: int, forced_recent: int = 0) -> np.ndarray:
+    """The k pages of largest score, by full sort; ties go to the lower page; the
+    last `forced_recent` pages are always in the set and count inside k. Output
+    ascending. score [n_pages]."""
+    n = score.shape[0]
+    if not (0 < k <= n) or not (0 <= forced_recent <= k):
+        raise ValueError("need 0 < k <= n_pages and 0 <= forced_recent <= k")
+    key = np.array(score, dtype=np.float64, copy=True)
+    if forced_recent:
+        key[n - forced_recent:] = np.inf
+    # stable sort of the negated key: equal keys stay in ascending page order
+    order = np.argsort(-key, kind="stable")
+    return np.sort(order[:k]).astype(np.int32)
+
+
+def select_topk(q_tok: np.ndarray, lm: np.ndarray, n_pages: np.ndarray, k: int,
+                forced_recent: int = 0, group_reduce: str = "softmax_max"):
+    """Per-KV-head critical set of every request (Sec. 2.2, Sec. 4.1).
+
+    q_tok [B, Hq, d], lm [B, Hkv, P, d], n_pages [B].
+    Returns (idx [B, Hkv, k] int32 ascending, scores: list of [Hkv, n_pages[b]])."""
+    B = q_tok.shape[0]
+    Hkv = lm.shape[1]
+    idx = np.empty((B, Hkv, k), dtype=np.int32)
+    scores = []
+    for b in range(B):
+        sc, _, _ = page_scores(q_tok[b], lm[b], int(n_pages[b]), group_reduce)
+        scores.append(sc)
+        for g in range(Hkv):
+            idx[b, g] = topk_pages(sc[g], k, forced_recent)
+    return idx, scores
+
+
+def gather_kv(kv_layer: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """Copy the selected pages into attention layout (Sec. 5.4 assembly; the bits
+    are unchanged). kv_layer [B, Hkv, P, 2, T, d] (any dtype), idx [B, Hkv, k]
+    → slot [B, Hkv, 2, k*T, d]."""
+    B, Hkv, P, two, T, d = kv_layer.shape
+    k = idx.shape[2]
+    slot = np.empty((B, Hkv, 2, k * T, d), dtype=kv_layer.dtype)
+    for b in range(B):
+        for g in range(Hkv):
+            for j in range(k):
+                p = int(idx[b, g, j])
+                slot[b, g, 0, j * T:(j + 1) * T, :] = kv_layer[b, g, p, 0]
+                slot[b, g, 1, j * T:(j + 1) * T, :] = kv_layer[b, g, p, 1]
+    return slot
+
+
+def sparse_decode_attn(q: np.ndarray, slot: np.ndarray, idx: np.ndarray, ctx_len: np.ndarray,
+                       page_tokens: int, return_weights: bool = False):
+    """Scaled-dot-product GQA attention of every query token over the gathered
+    set only (Sec. 4.2, Sec. 5.4: attention observes the layer's sparse KV set).
+
+    q [B, Tq, Hq, d]; slot [B, Hkv, 2, k*T, d]; idx [B, Hkv, k]; ctx_len [B].
+    Gathered token (j, i) sits at context position idx[j]*T + i and is masked
+    out when that position is >= ctx_len[b]. Both query tokens see the same set.
+    Returns (out [B, Tq, Hq, d] fp64, lse [B, Tq, Hq] fp64[, weights])."""
+    q = np.asarray(q, dtype=np.float64)
+    slot = np.asarray(slot, dtype=np.float64)
+    B, Tq, Hq, d = q.shape
+    Hkv = slot.shape[1]
+    G = Hq // Hkv
+    n_tok = slot.shape[3]
+    T = page_tokens
+    out = np.zeros((B, Tq, Hq, d), dtype=np.float64)
+    lse = np.zeros((B, Tq, Hq), dtype=np.float64)
+    weights = np.zeros((B, Tq, Hq, n_tok), dtype=np.float64) if return_weights else None
+    for b in range(B):
+        for g in range(Hkv):
+            pos = (idx[b, g].astype(np.int64)[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+            valid = pos < int(ctx_len[b])
+            keys = slot[b, g, 0]
+            vals = slot[b, g, 1]
+            for t in range(Tq):
+                for h in range(g * G, (g + 1) * G):
+                    z = keys @ q[b, t, h] / np.sqrt(float(d))
+                    z = np.where(valid, z, -np.inf)
+                    m = z.max()
+                    e = np.exp(z - m)
+                    den = e.sum()
+                    w = e / den
+                    out[b, t, h] = w @ vals
+                    lse[b, t, h] = m + np.log(den)
+                    if return_weights:
+                        weights[b, t, h] = w
+    if return_weights:
+        return out, lse, weights
+    return out, lse
+
+
+def decode_chain(q_init: np.ndarray, q_steps: np.ndarray, lm_layers, kv_layers, n_pages: np.ndarray,
+                 ctx_len: np.ndarray, k: int, page_tokens: int, forced_recent: int = 0):
+    """Several decode steps of every layer (Sec. 4.1, Sec. 5.2, Sec. 5.3):
+
+      idx[0][l]   = select(q_init[l])                      (stand-in for the pre-decode step)
+      out[t][l]   = attn(q_steps[t][l], gather(idx[t][l]))  (both tokens)
+      idx[t+1][l] = select(speculated token of q_steps[t][l])
+
+    q_init [L, B, Hq, d]; q_steps [S, L, B, 2, Hq, d]; lm_layers[l] [B, Hkv, P, d];
+    kv_layers[l] [B, Hkv, P, 2, T, d]. Returns (outs [S, L, B, 2, Hq, d], idxs [S+1, L, B, Hkv, k])."""
+    S, L = q_steps.shape[0], q_steps.shape[1]
+    B = q_steps.shape[2]
+    Hkv = lm_layers[0].shape[1]
+    idxs = np.empty((S + 1, L, B, Hkv, k), dtype=np.int32)
+    outs = np.empty(q_steps.shape, dtype=np.float64)
+    for l in range(L):
+        idxs[0, l], _ = select_topk(q_init[l], lm_layers[l], n_pages, k, forced_recent)
+    for t in range(S):
+        for l in range(L):
+            slot = gather_kv(kv_layers[l], idxs[t, l])
+            outs[t, l], _ = sparse_decode_attn(q_steps[t, l], slot, idxs[t, l], ctx_len, page_tokens)
+            idxs[t + 1, l], _ = select_topk(q_steps[t, l][:, 1], lm_layers[l], n_pages, k, forced_recent)
+    return outs, idxs
