@@ -1,0 +1,188 @@
+/* dd.h — C ABI of the sparse decode hot path (DualDecoder, arxiv 2607.26475), B200 / sm_100a.
+ *
+ * Per layer and request: score the KV pages from the speculated token's query against
+ * static GPU-resident page landmarks, pick a per-KV-head top-k set, gather those pages
+ * from pinned host memory into a layer-scoped ring slot on a side stream, and run GQA
+ * decode attention over the gathered set only.
+ *
+ * Conventions
+ *   - every function returns int: DD_OK (0) or a negative DD_ERR_* code; nothing throws,
+ *     aborts or traps. dd_last_error_message() gives the text of the last failure.
+ *   - "dev" pointers are CUDA device pointers of the context's device; "host" pointers are
+ *     ordinary host memory; "pinned" pointers are page-locked host memory the device can
+ *     read (cudaHostAlloc / cudaHostRegister; torch pin_memory). Pageable host memory is
+ *     rejected with DD_ERR_NOT_PINNED before any kernel is launched.
+ *   - the caller owns every tensor and both streams. The library owns the context, its
+ *     events, its scratch memory, its index tables and (unless supplied) the ring.
+ *   - all kernel entry points are asynchronous on the stream they are given (or on the
+ *     context's streams for the pipelined calls); dd_create, dd_destroy, dd_sync and
+ *     dd_device_error synchronise.
+ *   - the scratch memory of a context is shared by its calls: calls of the same kind must
+ *     be stream-ordered with respect to each other (the pipelined path does this itself).
+ *   - bf16 tensors are dense, row-major in the index order written, 16-byte aligned.
+ *   - geometry supported by the kernels: head_dim 128, page_tokens 16,
+ *     n_q_tokens * (n_q_heads / n_kv_heads) <= 8. Anything else is DD_ERR_INVALID_ARG.
+ *
+ * Notation: B requests, L layers, Hq query heads, Hkv KV heads, G = Hq/Hkv, d = head_dim,
+ * T = page_tokens, P = max_pages, k = k_pages, Tq = n_q_tokens (token 0 = current output
+ * token, token 1 = speculated token), D = ring_depth.
+ */
+#ifndef DD_H_
+#define DD_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DD_OK                 0
+#define DD_ERR_INVALID_ARG   (-1)
+#define DD_ERR_NOT_PINNED    (-2)
+#define DD_ERR_CUDA          (-3)
+#define DD_ERR_TIMEOUT       (-4)
+#define DD_ERR_INDEX_RANGE   (-5)   /* a page index outside [0, n_pages) reached a kernel; it was clamped */
+#define DD_ERR_STATE         (-6)   /* call out of order (not bound, not primed, wrong step/layer) */
+#define DD_ERR_WAIT_EXPIRED  (-7)   /* a bounded device-side wait gave up; the kernel returned early */
+
+#define DD_GATHER_LOADS  0          /* zero-copy: warps read the pinned pages with 16-byte loads */
+#define DD_GATHER_BULK   1          /* bulk-copy engine: pinned page -> shared memory -> slot (cp.async.bulk) */
+
+typedef struct dd_ctx dd_ctx;
+
+typedef struct dd_config {
+  int n_layers;              /* L */
+  int batch;                 /* B */
+  int n_q_heads;             /* Hq */
+  int n_kv_heads;            /* Hkv */
+  int head_dim;              /* d, must be 128 */
+  int page_tokens;           /* T, must be 16 */
+  int max_pages;             /* P: pages per request in the landmark and host-store layouts */
+  int k_pages;               /* k: selected pages per KV head (budget / T) */
+  int forced_recent_pages;   /* last pages of every request that are always selected; counted inside k */
+  int n_q_tokens;            /* Tq: 1 or 2 */
+  int ring_depth;            /* D >= 2 (2 = the two-buffer scheme) */
+  int gather_mode;           /* DD_GATHER_LOADS or DD_GATHER_BULK */
+  int gather_ctas;           /* thread blocks the gather may occupy; 0 = library default */
+  int attn_splits;           /* splits of the gathered set per (request, KV head); 0 = chosen from the SM count */
+  void* compute_stream;      /* cudaStream_t used by the pipelined calls for attention and selection */
+  void* copy_stream;         /* cudaStream_t used by the pipelined calls for the gather */
+  void* ring_mem;            /* optional caller-owned ring of dd_ring_bytes(); NULL = library allocates */
+  size_t ring_bytes;         /* size of ring_mem when supplied */
+} dd_config;
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Validates the configuration, allocates events, scratch, the index tables [2][L][B][Hkv][k]
+ * and (if ring_mem is NULL) the ring of D slots on the current device. */
+int dd_create(const dd_config* cfg, dd_ctx** out);
+/* Waits for the context's streams (bounded, 10 s) and frees what dd_create allocated. */
+int dd_destroy(dd_ctx* ctx);
+/* Bytes of one ring slot [B][Hkv][2][k*T][d] bf16, of the whole ring (D slots) and of the
+ * library's scratch for this configuration. 0 for an invalid configuration. */
+size_t dd_slot_bytes(const dd_config* cfg);
+size_t dd_ring_bytes(const dd_config* cfg);
+size_t dd_scratch_bytes(const dd_config* cfg);
+/* Device address of ring slot `slot` (0 <= slot < D). For tests and statistics. */
+int dd_slot_ptr(dd_ctx* ctx, int slot, void** dev_out);
+const char* dd_strerror(int code);
+const char* dd_last_error_message(dd_ctx* ctx);
+/* Synchronises the context's streams (bounded by timeout_s), then reads and clears the device
+ * error word. *code is DD_OK, DD_ERR_INDEX_RANGE or DD_ERR_WAIT_EXPIRED; *detail is the
+ * offending value (first bad index, or the id of the wait that gave up). */
+int dd_device_error(dd_ctx* ctx, double timeout_s, int* code, int* detail);
+/* Host wait on both context streams with a deadline: DD_ERR_TIMEOUT instead of hanging. */
+int dd_sync(dd_ctx* ctx, double timeout_s);
+
+/* ---- set-up step ---------------------------------------------------------------------------- */
+
+/* Landmarks of one layer (Sec. 2.2: adjacent KV entries are segmented into chunks with
+ * compressed landmarks; Sec. 4.1: built before decoding and fixed afterwards). Here a
+ * landmark is the mean of the valid keys of a page: fp32 sum in token order, fp32 divide,
+ * round-to-nearest-even to bf16; a page with no valid token gets zeros.
+ *   kv_layer   pinned or dev, bf16 [B][Hkv][P][2][T][d] ([..][0] = K, [..][1] = V)
+ *   ctx_len    dev int32 [B], tokens per request
+ *   landmarks  dev bf16 [B][Hkv][P][d], written */
+int dd_build_landmarks(dd_ctx* ctx, const void* kv_layer, const int* ctx_len, void* landmarks, void* stream);
+
+/* ---- the three kernels of the path ----------------------------------------------------------- */
+
+/* Retrieval index of one layer (Sec. 2.2, Sec. 4.1: the index is determined by the token's
+ * query and the GPU-resident landmarks; Sec. 4.1 "Retrieval index prediction": the speculated
+ * token's query predicts the next step's index).
+ *   s[h,p]     = <q[b,q_token,h,:], landmarks[b,h/G,p,:]> / sqrt(d)     for p < n_pages[b]
+ *   score[g,p] = max over the G heads of group g of softmax_p(s[h,:])[p]
+ * The last forced_recent_pages valid pages are always selected; the remaining k - forced are
+ * the highest scores among the others; equal scores go to the lower page.
+ *   q           dev bf16 [B][Tq][Hq][d]
+ *   q_token     which token's query scores (1 = speculated; 0 when Tq == 1)
+ *   landmarks   dev bf16 [B][Hkv][P][d] of this layer
+ *   n_pages     dev int32 [B], valid pages per request; k <= n_pages[b] <= P is required
+ *               (a violating request gets indices clamped into range and DD_ERR_INDEX_RANGE
+ *               in the device error word)
+ *   out_idx     dev int32 [B][Hkv][k], ascending page numbers, written
+ *   out_scores  dev fp32 [B][Hkv][P] or NULL; score[g,p] for p < n_pages[b], written */
+int dd_select_topk(dd_ctx* ctx, const void* q, int q_token, const void* landmarks, const int* n_pages,
+                   int* out_idx, float* out_scores, void* stream);
+
+/* Gather of the selected pages into a ring slot in attention layout (Sec. 5.3: predicted KV
+ * entries are prefetched from host memory; Sec. 5.4 "GPU-side sparse KV assembly": the GPU
+ * places them at their final attention layout). A bit copy:
+ *   slot[b][g][0|1][j*T + i][:] = host_kv_layer[b][g][idx[b][g][j]][0|1][i][:]
+ *   host_kv_layer  pinned (or dev) bf16 [B][Hkv][P][2][T][d] of this layer
+ *   idx            dev int32 [B][Hkv][k]
+ *   n_pages        dev int32 [B] or NULL; when given, idx outside [0, n_pages[b]) is clamped
+ *                  and reported (otherwise checked against P)
+ *   slot           ring slot number, 0 <= slot < D */
+int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, const int* idx, const int* n_pages,
+                           int slot, void* stream);
+
+/* GQA decode attention of every query token over the gathered set only (Sec. 4.2, Sec. 5.4:
+ * the attention kernel observes the layer's complete sparse KV set; Sec. 5.2: the output token
+ * and the speculated token are computed in one call). bf16 inputs, fp32 accumulation, bf16 out.
+ *   z[j,i]  = <q[b,t,h,:], Kslot[b,h/G,j*T+i,:]> / sqrt(d), dropped when idx[b,h/G,j]*T + i >= ctx_len[b]
+ *   out[b,t,h,:] = sum softmax(z) * Vslot
+ *   q        dev bf16 [B][Tq][Hq][d]
+ *   idx      dev int32 [B][Hkv][k] (the set the slot was gathered with; used for the mask only)
+ *   ctx_len  dev int32 [B]
+ *   out      dev bf16 [B][Tq][Hq][d], written
+ *   out_lse  dev fp32 [B][Tq][Hq] or NULL; natural-log sum of exp(z), written */
+int dd_sparse_decode_attn(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len,
+                          void* out, float* out_lse, void* stream);
+
+/* ---- the pipelined layer step ---------------------------------------------------------------- */
+
+/* Binds the per-layer tables used by dd_prime / dd_decode_layer_step.
+ *   landmarks_per_layer  host array of L dev pointers, each bf16 [B][Hkv][P][d]
+ *   host_kv_per_layer    host array of L pinned (or dev) pointers, each bf16 [B][Hkv][P][2][T][d]
+ *   n_pages, ctx_len     dev int32 [B]
+ * The arrays of pointers are copied; the tensors are not. */
+int dd_bind(dd_ctx* ctx, const void* const* landmarks_per_layer, const void* const* host_kv_per_layer,
+            const int* n_pages, const int* ctx_len);
+
+/* Priming selection for every layer — the stand-in for the pre-decoding step that yields the
+ * first speculated token (Sec. 5.2 "First speculative token initialization") — followed by the
+ * gathers of layers 0..min(D,L)-1 of step 0 on the copy stream.
+ *   q_init  dev bf16 [L][B][Hq][d] */
+int dd_prime(dd_ctx* ctx, const void* q_init);
+
+/* One layer of one decode step, in (step, layer) order starting at (0, 0) (Sec. 5.3 "Layer-aware
+ * KV transfer overlapping": the transfer for layer i+2 starts when the attention of layer i is
+ * done; Sec. 5.4 "Two-layer ping-pong buffering": the compute stream waits for the slot's
+ * transfer-complete event, the copy stream waits for the slot's buffer-released event):
+ *   compute stream: wait ready[slot(layer)] -> attention(step, layer) over the set selected one
+ *                   step earlier -> record released[slot] -> selection from q's speculated token
+ *                   -> index set of (step+1, layer)
+ *   copy stream:    wait released[slot] (and the selection it depends on) -> gather of layer
+ *                   layer+D of this step, or of layer layer+D-L of the next step
+ *   q    dev bf16 [B][Tq][Hq][d]
+ *   out  dev bf16 [B][Tq][Hq][d], written */
+int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out);
+
+/* Device address of the index set [B][Hkv][k] that attention uses at (step parity, layer). No copy. */
+int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* DD_H_ */

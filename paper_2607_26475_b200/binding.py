@@ -1,0 +1,215 @@
+"""Thin ctypes binding of the C-ABI library (`include/dd.h`): argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels. torch is used for device and
+pinned memory and for streams; tensors are passed as raw pointers. There is no CPU
+fallback: importing this module raises if `libdd.so` has not been built
+(`python -m paper_2607_26475_b200.build`).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdd.so")
+
+DD_OK = 0
+DD_ERR_INVALID_ARG = -1
+DD_ERR_NOT_PINNED = -2
+DD_ERR_CUDA = -3
+DD_ERR_TIMEOUT = -4
+DD_ERR_INDEX_RANGE = -5
+DD_ERR_STATE = -6
+DD_ERR_WAIT_EXPIRED = -7
+DD_GATHER_LOADS = 0
+DD_GATHER_BULK = 1
+
+EXPORTS = [
+    "dd_create", "dd_destroy", "dd_slot_bytes", "dd_ring_bytes", "dd_scratch_bytes", "dd_slot_ptr",
+    "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
+    "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
+    "dd_decode_layer_step", "dd_get_indices",
+]
+
+
+class DDConfig(C.Structure):
+    """Mirror of `dd_config`."""
+    _fields_ = [
+        ("n_layers", C.c_int), ("batch", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
+        ("head_dim", C.c_int), ("page_tokens", C.c_int), ("max_pages", C.c_int), ("k_pages", C.c_int),
+        ("forced_recent_pages", C.c_int), ("n_q_tokens", C.c_int), ("ring_depth", C.c_int),
+        ("gather_mode", C.c_int), ("gather_ctas", C.c_int), ("attn_splits", C.c_int),
+        ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
+        ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
+    ]
+
+
+class DDError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"dd error {code}: {message}")
+        self.code = code
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_26475_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = C.CDLL(LIB_PATH)
+    vp, ip = C.c_void_p, C.c_int
+    lib.dd_create.argtypes = [C.POINTER(DDConfig), C.POINTER(vp)]
+    lib.dd_destroy.argtypes = [vp]
+    for name in ("dd_slot_bytes", "dd_ring_bytes", "dd_scratch_bytes"):
+        getattr(lib, name).argtypes = [C.POINTER(DDConfig)]
+        getattr(lib, name).restype = C.c_size_t
+    lib.dd_slot_ptr.argtypes = [vp, ip, C.POINTER(vp)]
+    lib.dd_strerror.argtypes = [ip]
+    lib.dd_strerror.restype = C.c_char_p
+    lib.dd_last_error_message.argtypes = [vp]
+    lib.dd_last_error_message.restype = C.c_char_p
+    lib.dd_device_error.argtypes = [vp, C.c_double, C.POINTER(ip), C.POINTER(ip)]
+    lib.dd_sync.argtypes = [vp, C.c_double]
+    lib.dd_build_landmarks.argtypes = [vp, vp, vp, vp, vp]
+    lib.dd_select_topk.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
+    lib.dd_gather_kv_from_host.argtypes = [vp, vp, vp, vp, ip, vp]
+    lib.dd_sparse_decode_attn.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp]
+    lib.dd_bind.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp]
+    lib.dd_prime.argtypes = [vp, vp]
+    lib.dd_decode_layer_step.argtypes = [vp, ip, ip, vp, vp]
+    lib.dd_get_indices.argtypes = [vp, ip, ip, C.POINTER(vp)]
+    return lib
+
+
+lib = _load()
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(s) -> int:
+    if s is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+class Context:
+    """Owns one `dd_ctx`. Method names follow the C entry points (without the `dd_` prefix)."""
+
+    def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                 page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
+                 gather_ctas=0, attn_splits=0, compute_stream=None, copy_stream=None, ring=None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
+        self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
+        self.copy_stream = copy_stream if copy_stream is not None else torch.cuda.Stream()
+        self._ring = ring
+        self.cfg = DDConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, page_tokens, max_pages, k_pages,
+                            forced_recent_pages, n_q_tokens, ring_depth, gather_mode, gather_ctas, attn_splits,
+                            self.compute_stream.cuda_stream, self.copy_stream.cuda_stream,
+                            _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0)
+        self._h = C.c_void_p()
+        self._keep = []
+        rc = lib.dd_create(C.byref(self.cfg), C.byref(self._h))
+        if rc != DD_OK:
+            raise DDError(rc, lib.dd_last_error_message(None).decode())
+
+    # -- plumbing
+    def _check(self, rc: int):
+        if rc != DD_OK:
+            raise DDError(rc, lib.dd_last_error_message(self._h).decode())
+
+    def close(self):
+        if self._h:
+            rc = lib.dd_destroy(self._h)
+            self._h = C.c_void_p()
+            if rc != DD_OK:
+                raise DDError(rc, "dd_destroy failed")
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def slot_bytes(self) -> int:
+        return lib.dd_slot_bytes(C.byref(self.cfg))
+
+    def ring_bytes(self) -> int:
+        return lib.dd_ring_bytes(C.byref(self.cfg))
+
+    def scratch_bytes(self) -> int:
+        return lib.dd_scratch_bytes(C.byref(self.cfg))
+
+    def slot_ptr(self, slot: int) -> int:
+        p = C.c_void_p()
+        self._check(lib.dd_slot_ptr(self._h, slot, C.byref(p)))
+        return p.value
+
+    def slot_tensor(self, slot: int) -> torch.Tensor:
+        """A copy of ring slot `slot` as [B, Hkv, 2, k*T, d] bf16 (synchronises; for tests)."""
+        c = self.cfg
+        shape = (c.batch, c.n_kv_heads, 2, c.k_pages * c.page_tokens, c.head_dim)
+        out = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
+        torch.cuda.synchronize()
+        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), self.slot_ptr(slot), self.slot_bytes(), 3)
+        if int(rc) != 0:
+            raise RuntimeError(f"cudaMemcpy failed: {rc}")
+        return out
+
+    def sync(self, timeout_s: float = 60.0):
+        self._check(lib.dd_sync(self._h, timeout_s))
+
+    def device_error(self, timeout_s: float = 60.0):
+        code, detail = C.c_int(), C.c_int()
+        self._check(lib.dd_device_error(self._h, timeout_s, C.byref(code), C.byref(detail)))
+        return code.value, detail.value
+
+    # -- entry points
+    def build_landmarks(self, kv_layer, ctx_len, landmarks, stream=None):
+        self._check(lib.dd_build_landmarks(self._h, _ptr(kv_layer), _ptr(ctx_len), _ptr(landmarks), _stream(stream)))
+
+    def select_topk(self, q, q_token, landmarks, n_pages, out_idx, out_scores=None, stream=None):
+        self._check(lib.dd_select_topk(self._h, _ptr(q), q_token, _ptr(landmarks), _ptr(n_pages), _ptr(out_idx),
+                                       _ptr(out_scores), _stream(stream)))
+
+    def gather_kv_from_host(self, host_kv_layer, idx, n_pages, slot, stream=None):
+        self._check(lib.dd_gather_kv_from_host(self._h, _ptr(host_kv_layer), _ptr(idx), _ptr(n_pages), slot,
+                                               _stream(stream)))
+
+    def sparse_decode_attn(self, q, slot, idx, ctx_len, out, out_lse=None, stream=None):
+        self._check(lib.dd_sparse_decode_attn(self._h, _ptr(q), slot, _ptr(idx), _ptr(ctx_len), _ptr(out),
+                                              _ptr(out_lse), _stream(stream)))
+
+    def bind(self, landmarks_per_layer, host_kv_per_layer, n_pages, ctx_len):
+        L = self.cfg.n_layers
+        assert len(landmarks_per_layer) == L and len(host_kv_per_layer) == L
+        self._keep = [landmarks_per_layer, host_kv_per_layer, n_pages, ctx_len]    # keep the tensors alive
+        lm = (C.c_void_p * L)(*[_ptr(t) for t in landmarks_per_layer])
+        kv = (C.c_void_p * L)(*[_ptr(t) for t in host_kv_per_layer])
+        self._check(lib.dd_bind(self._h, lm, kv, _ptr(n_pages), _ptr(ctx_len)))
+
+    def prime(self, q_init):
+        self._check(lib.dd_prime(self._h, _ptr(q_init)))
+
+    def decode_layer_step(self, step, layer, q, out):
+        self._check(lib.dd_decode_layer_step(self._h, step, layer, _ptr(q), _ptr(out)))
+
+    def get_indices(self, step_parity, layer) -> torch.Tensor:
+        """A copy of the index set [B, Hkv, k] int32 used at (step parity, layer) (synchronises)."""
+        p = C.c_void_p()
+        self._check(lib.dd_get_indices(self._h, step_parity, layer, C.byref(p)))
+        c = self.cfg
+        out = torch.empty((c.batch, c.n_kv_heads, c.k_pages), dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p.value, out.numel() * 4, 3)
+        if int(rc) != 0:
+            raise RuntimeError(f"cudaMemcpy failed: {rc}")
+        return out

@@ -1,0 +1,464 @@
+// Host side of the C ABI: context life cycle, argument checks, and the layer-scoped ring with its
+// event protocol (transfer-complete / buffer-released) driving the pipelined layer step.
+#include <stdarg.h>
+#include <string.h>
+
+#include <chrono>
+#include <new>
+#include <thread>
+
+#include "dd_common.cuh"
+
+int dd_select_setup(dd_ctx* ctx);
+int dd_gather_setup(dd_ctx* ctx);
+
+static thread_local char g_errmsg[512] = "";
+
+int dd_fail(dd_ctx* ctx, int code, const char* fmt, ...) {
+  char* dst = ctx ? ctx->errmsg : g_errmsg;
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(dst, 512, fmt, ap);
+  va_end(ap);
+  if (ctx) memcpy(g_errmsg, ctx->errmsg, 512);
+  return code;
+}
+
+extern "C" const char* dd_strerror(int code) {
+  switch (code) {
+    case DD_OK: return "ok";
+    case DD_ERR_INVALID_ARG: return "invalid argument";
+    case DD_ERR_NOT_PINNED: return "host memory is not page-locked";
+    case DD_ERR_CUDA: return "CUDA error";
+    case DD_ERR_TIMEOUT: return "timed out";
+    case DD_ERR_INDEX_RANGE: return "page index out of range (clamped)";
+    case DD_ERR_STATE: return "call out of order";
+    case DD_ERR_WAIT_EXPIRED: return "a bounded device-side wait expired";
+    default: return "unknown error";
+  }
+}
+
+extern "C" const char* dd_last_error_message(dd_ctx* ctx) { return ctx ? ctx->errmsg : g_errmsg; }
+
+// ---------------------------------------------------------------------------------------------
+// configuration
+// ---------------------------------------------------------------------------------------------
+static const char* dd_check_config(const dd_config* c) {
+  if (!c) return "config is NULL";
+  if (c->head_dim != DD_D) return "head_dim must be 128";
+  if (c->page_tokens != DD_T) return "page_tokens must be 16";
+  if (c->n_layers < 1 || c->batch < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return "sizes must be positive";
+  if (c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a multiple of n_kv_heads";
+  if (c->n_q_tokens < 1 || c->n_q_tokens > 2) return "n_q_tokens must be 1 or 2";
+  if (c->n_q_tokens * (c->n_q_heads / c->n_kv_heads) > 8) return "n_q_tokens * group size must be <= 8";
+  if (c->max_pages < 1) return "max_pages must be positive";
+  if (c->k_pages < 1 || c->k_pages > c->max_pages) return "need 1 <= k_pages <= max_pages";
+  if (c->forced_recent_pages < 0 || c->forced_recent_pages > c->k_pages) return "need 0 <= forced_recent_pages <= k_pages";
+  if (c->ring_depth < 2 || c->ring_depth > DD_MAX_RING) return "ring_depth must be in [2, 8]";
+  if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK) return "unknown gather_mode";
+  if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
+  if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
+  if ((long long)c->batch * c->n_kv_heads * c->max_pages > 0x7fffffffLL) return "too many pages";
+  return nullptr;
+}
+
+static int dd_resolve_splits(const dd_config* c, int sm_count) {
+  int S = c->attn_splits;
+  if (S <= 0) {
+    // enough blocks for about four per SM, but at least four pages (one per warp) in a split
+    const int problems = c->batch * c->n_kv_heads;
+    S = (4 * sm_count + problems - 1) / problems;
+    const int s_max = c->k_pages / 4 > 0 ? c->k_pages / 4 : 1;
+    if (S > s_max) S = s_max;
+    if (S > 64) S = 64;
+  }
+  if (S > c->k_pages) S = c->k_pages;
+  if (S < 1) S = 1;
+  return S;
+}
+
+struct dd_sizes {
+  size_t score_s, score_part, topk_keys, part_o, part_ml, ticket, idx_tab, err;
+  size_t total() const { return score_s + score_part + topk_keys + part_o + part_ml + ticket + idx_tab + err; }
+};
+
+static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
+  dd_sizes z;
+  const size_t B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads, P = c->max_pages;
+  const size_t G = Hq / Hkv, tiles = (P + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
+  z.score_s = up256(B * Hkv * P * G * 4);
+  z.score_part = up256(B * Hq * tiles * 8);
+  z.topk_keys = up256(B * Hkv * P * 4);
+  z.part_o = up256(B * Hkv * (size_t)S * 8 * DD_D * 4);
+  z.part_ml = up256(B * Hkv * (size_t)S * 8 * 8);
+  z.ticket = up256(B * Hkv * 4);
+  z.idx_tab = up256((size_t)2 * c->n_layers * B * Hkv * c->k_pages * 4);
+  z.err = 256;
+  return z;
+}
+
+static int dd_sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+  return sms;
+}
+
+extern "C" size_t dd_slot_bytes(const dd_config* c) {
+  if (dd_check_config(c)) return 0;
+  return (size_t)c->batch * c->n_kv_heads * c->k_pages * DD_PAGE_BYTES;
+}
+extern "C" size_t dd_ring_bytes(const dd_config* c) { return dd_slot_bytes(c) * (c ? (size_t)c->ring_depth : 0); }
+extern "C" size_t dd_scratch_bytes(const dd_config* c) {
+  if (dd_check_config(c)) return 0;
+  return dd_compute_sizes(c, dd_resolve_splits(c, dd_sm_count())).total();
+}
+
+// ---------------------------------------------------------------------------------------------
+// life cycle
+// ---------------------------------------------------------------------------------------------
+static void dd_free_all(dd_ctx* ctx) {
+  if (ctx->score_s) cudaFree(ctx->score_s);      // one allocation holds all the scratch
+  if (ctx->own_ring && ctx->ring) cudaFree(ctx->ring);
+  for (int i = 0; i < DD_MAX_RING; ++i) {
+    if (ctx->ready[i]) cudaEventDestroy(ctx->ready[i]);
+    if (ctx->released[i]) cudaEventDestroy(ctx->released[i]);
+  }
+  if (ctx->sel_done) {
+    for (int l = 0; l < ctx->cfg.n_layers; ++l)
+      if (ctx->sel_done[l]) cudaEventDestroy(ctx->sel_done[l]);
+    delete[] ctx->sel_done;
+  }
+  delete[] ctx->landmarks;
+  delete[] ctx->host_kv;
+  delete ctx;
+}
+
+extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
+  if (!out) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: out is NULL");
+  *out = nullptr;
+  if (const char* why = dd_check_config(cfg)) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: %s", why);
+  dd_ctx* ctx = new (std::nothrow) dd_ctx();
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: out of host memory");
+  memset(ctx, 0, sizeof(*ctx));
+  ctx->cfg = *cfg;
+  cudaError_t e = cudaGetDevice(&ctx->device);
+  if (e != cudaSuccess) {
+    int rc = dd_fail(nullptr, DD_ERR_CUDA, "dd_create: no CUDA device: %s", cudaGetErrorString(e));
+    delete ctx;
+    return rc;
+  }
+  ctx->sm_count = dd_sm_count();
+  ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->n_rows = cfg->n_q_tokens * ctx->G;
+  ctx->score_tiles = (cfg->max_pages + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
+  ctx->attn_splits = dd_resolve_splits(cfg, ctx->sm_count);
+  ctx->slot_bytes = dd_slot_bytes(cfg);
+  const dd_sizes z = dd_compute_sizes(cfg, ctx->attn_splits);
+
+#define DD_CREATE_TRY(expr)                                                                        \
+  do {                                                                                             \
+    cudaError_t e__ = (expr);                                                                      \
+    if (e__ != cudaSuccess) {                                                                      \
+      int rc__ = dd_fail(nullptr, DD_ERR_CUDA, "dd_create: %s: %s", #expr, cudaGetErrorString(e__)); \
+      dd_free_all(ctx);                                                                            \
+      return rc__;                                                                                 \
+    }                                                                                              \
+  } while (0)
+
+  char* base = nullptr;
+  DD_CREATE_TRY(cudaMalloc(&base, z.total()));
+  ctx->score_s = (float*)base;                       base += z.score_s;
+  ctx->score_part = (float2*)base;                   base += z.score_part;
+  ctx->topk_keys = (uint32_t*)base;                  base += z.topk_keys;
+  ctx->attn_part_o = (float*)base;                   base += z.part_o;
+  ctx->attn_part_ml = (float2*)base;                 base += z.part_ml;
+  ctx->attn_ticket = (unsigned int*)base;            base += z.ticket;
+  ctx->idx_tab = (int*)base;                         base += z.idx_tab;
+  ctx->err_word = (int*)base;
+  DD_CREATE_TRY(cudaMemset(ctx->attn_ticket, 0, z.ticket));
+  DD_CREATE_TRY(cudaMemset(ctx->idx_tab, 0, z.idx_tab));
+  DD_CREATE_TRY(cudaMemset(ctx->err_word, 0, z.err));
+  if (cfg->ring_mem) {
+    if (cfg->ring_bytes < dd_ring_bytes(cfg)) {
+      int rc = dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: ring_mem holds %zu bytes, %zu needed", cfg->ring_bytes,
+                       dd_ring_bytes(cfg));
+      dd_free_all(ctx);
+      return rc;
+    }
+    if (((uintptr_t)cfg->ring_mem) & 15) {
+      int rc = dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: ring_mem must be 16-byte aligned");
+      dd_free_all(ctx);
+      return rc;
+    }
+    ctx->ring = (char*)cfg->ring_mem;
+  } else {
+    DD_CREATE_TRY(cudaMalloc(&ctx->ring, dd_ring_bytes(cfg)));
+    ctx->own_ring = true;
+  }
+  for (int i = 0; i < cfg->ring_depth; ++i) {
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->ready[i], cudaEventDisableTiming));
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->released[i], cudaEventDisableTiming));
+  }
+  ctx->sel_done = new cudaEvent_t[cfg->n_layers]();
+  for (int l = 0; l < cfg->n_layers; ++l)
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->sel_done[l], cudaEventDisableTiming));
+  ctx->landmarks = new const void*[cfg->n_layers]();
+  ctx->host_kv = new const void*[cfg->n_layers]();
+  int rc = dd_select_setup(ctx);
+  if (rc == DD_OK) rc = dd_gather_setup(ctx);
+  if (rc != DD_OK) {
+    memcpy(g_errmsg, ctx->errmsg, 512);
+    dd_free_all(ctx);
+    return rc;
+  }
+  DD_CREATE_TRY(cudaDeviceSynchronize());
+#undef DD_CREATE_TRY
+  *out = ctx;
+  return DD_OK;
+}
+
+extern "C" int dd_sync(dd_ctx* ctx, double timeout_s) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sync: ctx is NULL");
+  const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(timeout_s);
+  cudaStream_t streams[2] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream};
+  for (int i = 0; i < 2; ++i) {
+    for (;;) {
+      cudaError_t e = cudaStreamQuery(streams[i]);
+      if (e == cudaSuccess) break;
+      if (e != cudaErrorNotReady) return dd_fail(ctx, DD_ERR_CUDA, "dd_sync: %s", cudaGetErrorString(e));
+      if (std::chrono::steady_clock::now() > deadline)
+        return dd_fail(ctx, DD_ERR_TIMEOUT, "dd_sync: streams still busy after %.3f s", timeout_s);
+      std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+  }
+  return DD_OK;
+}
+
+extern "C" int dd_destroy(dd_ctx* ctx) {
+  if (!ctx) return DD_OK;
+  int rc = dd_sync(ctx, 10.0);
+  if (rc == DD_ERR_TIMEOUT) return rc;             // memory still in use by the device: leak rather than free
+  dd_free_all(ctx);
+  return DD_OK;
+}
+
+extern "C" int dd_device_error(dd_ctx* ctx, double timeout_s, int* code, int* detail) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_device_error: ctx is NULL");
+  int rc = dd_sync(ctx, timeout_s);
+  if (rc != DD_OK) return rc;
+  int w[2] = {0, 0};
+  DD_CUDA_TRY(ctx, cudaDeviceSynchronize());       // standalone calls may have used other streams
+  DD_CUDA_TRY(ctx, cudaMemcpy(w, ctx->err_word, sizeof(w), cudaMemcpyDeviceToHost));
+  DD_CUDA_TRY(ctx, cudaMemset(ctx->err_word, 0, sizeof(w)));
+  if (code) *code = w[0];
+  if (detail) *detail = w[1];
+  return DD_OK;
+}
+
+extern "C" int dd_slot_ptr(dd_ctx* ctx, int slot, void** dev_out) {
+  if (!ctx || !dev_out) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_slot_ptr: NULL argument");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_slot_ptr: slot %d of %d", slot, ctx->cfg.ring_depth);
+  *dev_out = ctx->ring + (size_t)slot * ctx->slot_bytes;
+  return DD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// pointer checks
+// ---------------------------------------------------------------------------------------------
+// Device pointer of the context's device (16-byte aligned), or failure.
+static int dd_check_dev(dd_ctx* ctx, const void* p, const char* what) {
+  if (!p) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is NULL", what);
+  if (((uintptr_t)p) & 15) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is not 16-byte aligned", what);
+  cudaPointerAttributes a;
+  cudaError_t e = cudaPointerGetAttributes(&a, p);
+  if (e != cudaSuccess) { cudaGetLastError(); return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s: %s", what, cudaGetErrorString(e)); }
+  if (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is not device memory", what);
+  if (a.type == cudaMemoryTypeDevice && a.device != ctx->device)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s lives on device %d, the context on %d", what, a.device, ctx->device);
+  return DD_OK;
+}
+
+// Page-locked host memory (or device memory): returns the address the device uses.
+static int dd_check_store(dd_ctx* ctx, const void* p, const char* what, const void** dev_visible) {
+  if (!p) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is NULL", what);
+  if (((uintptr_t)p) & 15) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is not 16-byte aligned", what);
+  cudaPointerAttributes a;
+  cudaError_t e = cudaPointerGetAttributes(&a, p);
+  if (e != cudaSuccess) { cudaGetLastError(); return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s: %s", what, cudaGetErrorString(e)); }
+  if (a.type == cudaMemoryTypeUnregistered)
+    return dd_fail(ctx, DD_ERR_NOT_PINNED, "%s is pageable host memory; page-lock it (cudaHostAlloc / cudaHostRegister)", what);
+  if (a.type == cudaMemoryTypeHost) {
+    if (!a.devicePointer) return dd_fail(ctx, DD_ERR_NOT_PINNED, "%s is page-locked but not mapped into the device", what);
+    *dev_visible = a.devicePointer;
+    return DD_OK;
+  }
+  if (a.type == cudaMemoryTypeDevice && a.device != ctx->device)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s lives on device %d, the context on %d", what, a.device, ctx->device);
+  *dev_visible = p;
+  return DD_OK;
+}
+
+#define DD_TRY(expr)             \
+  do {                           \
+    int rc__ = (expr);           \
+    if (rc__ != DD_OK) return rc__; \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// stand-alone entry points
+// ---------------------------------------------------------------------------------------------
+extern "C" int dd_build_landmarks(dd_ctx* ctx, const void* kv_layer, const int* ctx_len, void* landmarks, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_build_landmarks: ctx is NULL");
+  const void* kv_dev = nullptr;
+  DD_TRY(dd_check_store(ctx, kv_layer, "kv_layer", &kv_dev));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
+  return dd_launch_build_landmarks(ctx, kv_dev, ctx_len, landmarks, (cudaStream_t)stream);
+}
+
+extern "C" int dd_select_topk(dd_ctx* ctx, const void* q, int q_token, const void* landmarks, const int* n_pages,
+                              int* out_idx, float* out_scores, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_select_topk: ctx is NULL");
+  if (q_token < 0 || q_token >= ctx->cfg.n_q_tokens)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "q_token %d outside [0, %d)", q_token, ctx->cfg.n_q_tokens);
+  DD_TRY(dd_check_dev(ctx, q, "q"));
+  DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
+  DD_TRY(dd_check_dev(ctx, out_idx, "out_idx"));
+  if (out_scores) DD_TRY(dd_check_dev(ctx, out_scores, "out_scores"));
+  return dd_launch_select(ctx, q, q_token, ctx->cfg.n_q_tokens, landmarks, n_pages, out_idx, out_scores,
+                          (cudaStream_t)stream);
+}
+
+extern "C" int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, const int* idx, const int* n_pages,
+                                      int slot, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_gather_kv_from_host: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  const void* kv_dev = nullptr;
+  DD_TRY(dd_check_store(ctx, host_kv_layer, "host_kv_layer", &kv_dev));
+  DD_TRY(dd_check_dev(ctx, idx, "idx"));
+  if (n_pages) DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
+  return dd_launch_gather(ctx, kv_dev, idx, n_pages, ctx->ring + (size_t)slot * ctx->slot_bytes, (cudaStream_t)stream);
+}
+
+extern "C" int dd_sparse_decode_attn(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len,
+                                     void* out, float* out_lse, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  DD_TRY(dd_check_dev(ctx, q, "q"));
+  DD_TRY(dd_check_dev(ctx, idx, "idx"));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  DD_TRY(dd_check_dev(ctx, out, "out"));
+  if (out_lse) DD_TRY(dd_check_dev(ctx, out_lse, "out_lse"));
+  return dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, idx, ctx_len, out, out_lse,
+                        (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// pipelined path
+// ---------------------------------------------------------------------------------------------
+extern "C" int dd_bind(dd_ctx* ctx, const void* const* landmarks_per_layer, const void* const* host_kv_per_layer,
+                       const int* n_pages, const int* ctx_len) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_bind: ctx is NULL");
+  if (!landmarks_per_layer || !host_kv_per_layer) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_bind: table is NULL");
+  ctx->bound = false;
+  ctx->primed = false;
+  for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+    DD_TRY(dd_check_dev(ctx, landmarks_per_layer[l], "landmarks_per_layer[l]"));
+    const void* dv = nullptr;
+    DD_TRY(dd_check_store(ctx, host_kv_per_layer[l], "host_kv_per_layer[l]", &dv));
+    ctx->landmarks[l] = landmarks_per_layer[l];
+    ctx->host_kv[l] = dv;
+  }
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  ctx->n_pages = n_pages;
+  ctx->ctx_len = ctx_len;
+  ctx->bound = true;
+  return DD_OK;
+}
+
+static int* dd_idx_of(dd_ctx* ctx, int parity, int layer) {
+  const dd_config& c = ctx->cfg;
+  return ctx->idx_tab + ((size_t)(parity & 1) * c.n_layers + layer) * c.batch * c.n_kv_heads * c.k_pages;
+}
+
+// Gather number n = step * L + layer goes to slot n % D. It may start once the attention that last
+// read the slot has released it and the selection that produced its index set is done.
+static int dd_enqueue_gather(dd_ctx* ctx, long long n) {
+  const dd_config& c = ctx->cfg;
+  const int layer = (int)(n % c.n_layers), step = (int)(n / c.n_layers);
+  const int slot = (int)(n % c.ring_depth);
+  cudaStream_t xs = (cudaStream_t)c.copy_stream;
+  if (ctx->released_recorded[slot]) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->released[slot], 0));
+  DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->sel_done[layer], 0));
+  DD_TRY(dd_launch_gather(ctx, ctx->host_kv[layer], dd_idx_of(ctx, step, layer), ctx->n_pages,
+                          ctx->ring + (size_t)slot * ctx->slot_bytes, xs));
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->ready[slot], xs));
+  return DD_OK;
+}
+
+extern "C" int dd_prime(dd_ctx* ctx, const void* q_init) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_prime: ctx is NULL");
+  if (!ctx->bound) return dd_fail(ctx, DD_ERR_STATE, "dd_prime: call dd_bind first");
+  DD_TRY(dd_check_dev(ctx, q_init, "q_init"));
+  const dd_config& c = ctx->cfg;
+  cudaStream_t cs = (cudaStream_t)c.compute_stream;
+  // a restart must not overtake work of an earlier run that still uses the ring or the index tables
+  DD_TRY(dd_sync(ctx, 30.0));
+  const size_t q_layer = (size_t)c.batch * c.n_q_heads * DD_D;
+  for (int l = 0; l < c.n_layers; ++l) {
+    DD_TRY(dd_launch_select(ctx, (const __nv_bfloat16*)q_init + l * q_layer, 0, 1, ctx->landmarks[l], ctx->n_pages,
+                            dd_idx_of(ctx, 0, l), nullptr, cs));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[l], cs));
+  }
+  for (int i = 0; i < DD_MAX_RING; ++i) ctx->released_recorded[i] = false;
+  const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
+  for (long long n = 0; n < ahead; ++n) DD_TRY(dd_enqueue_gather(ctx, n));
+  ctx->next_call = 0;
+  ctx->primed = true;
+  return DD_OK;
+}
+
+extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_decode_layer_step: ctx is NULL");
+  if (!ctx->primed) return dd_fail(ctx, DD_ERR_STATE, "dd_decode_layer_step: call dd_bind and dd_prime first");
+  const dd_config& c = ctx->cfg;
+  if (layer < 0 || layer >= c.n_layers || step < 0) return dd_fail(ctx, DD_ERR_INVALID_ARG, "bad (step, layer) = (%d, %d)", step, layer);
+  const long long n = (long long)step * c.n_layers + layer;
+  if (n != ctx->next_call)
+    return dd_fail(ctx, DD_ERR_STATE, "expected (step, layer) = (%lld, %lld), got (%d, %d)", ctx->next_call / c.n_layers,
+                   ctx->next_call % c.n_layers, step, layer);
+  DD_TRY(dd_check_dev(ctx, q, "q"));
+  DD_TRY(dd_check_dev(ctx, out, "out"));
+  cudaStream_t cs = (cudaStream_t)c.compute_stream;
+  const int slot = (int)(n % c.ring_depth);
+
+  DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));                    // transfer complete
+  DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, dd_idx_of(ctx, step, layer), ctx->ctx_len,
+                        out, nullptr, cs));
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
+  ctx->released_recorded[slot] = true;
+  DD_TRY(dd_launch_select(ctx, q, c.n_q_tokens - 1, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
+                          dd_idx_of(ctx, step + 1, layer), nullptr, cs));
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+  // the slot just released takes the gather `ahead` layers further on (index set known: it was
+  // selected one step earlier, or just now when the ring is deeper than the model)
+  const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
+  DD_TRY(dd_enqueue_gather(ctx, n + ahead));
+  ctx->next_call = n + 1;
+  return DD_OK;
+}
+
+extern "C" int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx) {
+  if (!ctx || !dev_idx) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_get_indices: NULL argument");
+  if (layer < 0 || layer >= ctx->cfg.n_layers) return dd_fail(ctx, DD_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
+  *dev_idx = dd_idx_of(ctx, step_parity, layer);
+  return DD_OK;
+}

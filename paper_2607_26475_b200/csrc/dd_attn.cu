@@ -1,0 +1,258 @@
+// GQA decode attention over the gathered set of a ring slot.
+//
+// Work is split flash-decoding style: grid (split, KV head, request), 4 warps per block, each warp
+// walks pages of its split with a running soft-max; the block merges its warps, and the last block of
+// a (request, KV head) to arrive merges the splits (arrival counter, no waiting).
+//
+// Both products run on warp-level bf16 MMAs in their transposed form, so that the up-to-8 query rows
+// that share a KV head (Tq tokens x G heads) are the N = 8 columns and nothing is padded:
+//   S^T[token, n] = K[token, :] . q[n, :]        A = K page (16 tokens x 128), B = q^T
+//   O^T[d, n]    += V^T[d, token] P^T[token, n]   A = V^T (16 channels x 16 tokens), B = P^T
+// K and V are read straight from global memory into MMA fragments with 16-byte loads:
+//   * for S^T the 128 channels may be summed in any order, so a thread feeds k-slots {2t,2t+1,2t+8,2t+9}
+//     of two consecutive k-steps with 8 consecutive channels of its token row (one load);
+//   * for O^T the rows of the MMA (channels) may be assigned freely, so a thread takes 8 consecutive
+//     channels of tokens 2t, 2t+1, 2t+8, 2t+9 and pairs neighbouring tokens with byte permutes;
+//   * P^T goes from accumulator layout to B-operand layout with one 8x8 matrix transpose per half page.
+#include "dd_common.cuh"
+
+constexpr int ATTN_WARPS = 4;
+constexpr int ATTN_THREADS = ATTN_WARPS * 32;
+constexpr int ATTN_ROWS = 8;       // query rows per KV head the MMA shape carries
+
+__device__ __forceinline__ uint32_t dd_movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+__device__ __forceinline__ uint32_t dd_pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
+    const __nv_bfloat16* __restrict__ q, const char* __restrict__ slot, const int* __restrict__ idx,
+    const int* __restrict__ ctx_len, __nv_bfloat16* __restrict__ out, float* __restrict__ out_lse,
+    float* __restrict__ part_o, float2* __restrict__ part_ml, unsigned int* __restrict__ ticket, int Hkv, int G, int Tq,
+    int k, int n_splits, int pages_per_split) {
+  const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const int Hq = Hkv * G;
+  const int n_rows = Tq * G;
+  const size_t bg = (size_t)b * Hkv + g;
+
+  __shared__ float sm_o[ATTN_WARPS][ATTN_ROWS][DD_D];
+  __shared__ float2 sm_ml[ATTN_WARPS][ATTN_ROWS];
+  __shared__ float sm_scale[ATTN_WARPS][ATTN_ROWS];
+  __shared__ int sm_last;
+
+  // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G)
+  uint4 qf[4];
+  if (gl < n_rows) {
+    const int tq = gl / G, hh = gl - tq * G;
+    const uint4* qrow =
+        reinterpret_cast<const uint4*>(q + (((size_t)b * Tq + tq) * Hq + g * G + hh) * DD_D);
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) qf[kk] = __ldg(qrow + kk * 4 + t);
+  } else {
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) qf[kk] = make_uint4(0u, 0u, 0u, 0u);
+  }
+
+  const char* kbase = slot + bg * 2 * (size_t)k * DD_HALF_PAGE_BYTES;
+  const char* vbase = kbase + (size_t)k * DD_HALF_PAGE_BYTES;
+  const int* idx_bg = idx + bg * k;
+  const int n_ctx = ctx_len[b];
+  const float scale_log2 = rsqrtf((float)DD_D) * 1.4426950408889634f;
+
+  float o[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  float m_run[2] = {-INFINITY, -INFINITY};   // columns n = 2t, 2t+1, log2 domain
+  float l_run[2] = {0.f, 0.f};               // partial over this lane's tokens
+
+  const int p_begin = split * pages_per_split;
+  const int p_end = min(k, p_begin + pages_per_split);
+  for (int j = p_begin + warp; j < p_end; j += ATTN_WARPS) {
+    // ---- loads: K rows gl and gl+8; V tokens 2t, 2t+1, 2t+8, 2t+9, channels [8gl, 8gl+8) and [64+8gl, ..)
+    const char* kp = kbase + (size_t)j * DD_HALF_PAGE_BYTES;
+    const char* vp = vbase + (size_t)j * DD_HALF_PAGE_BYTES;
+    uint4 klo[4], khi[4];
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      klo[kk] = dd_ld_stream(kp + gl * DD_ROW_BYTES + (kk * 4 + t) * 16);
+      khi[kk] = dd_ld_stream(kp + (gl + 8) * DD_ROW_BYTES + (kk * 4 + t) * 16);
+    }
+    uint32_t v[4][2][4];
+#pragma unroll
+    for (int tk = 0; tk < 4; ++tk) {
+      const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const uint4 w = dd_ld_stream(vp + tok * DD_ROW_BYTES + (c * 64 + gl * 8) * 2);
+        v[tk][c][0] = w.x; v[tk][c][1] = w.y; v[tk][c][2] = w.z; v[tk][c][3] = w.w;
+      }
+    }
+    const int page = idx_bg[j];
+
+    // ---- S^T = K q^T
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      dd_mma_bf16(acc, klo[kk].x, khi[kk].x, klo[kk].y, khi[kk].y, qf[kk].x, qf[kk].y);
+      dd_mma_bf16(acc, klo[kk].z, khi[kk].z, klo[kk].w, khi[kk].w, qf[kk].z, qf[kk].w);
+    }
+    // acc[0], acc[1]: token gl, columns 2t, 2t+1; acc[2], acc[3]: token gl+8
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] *= scale_log2;
+    if (page * DD_T + DD_T > n_ctx) {            // only the last page of a request can be partial
+      if (page * DD_T + gl >= n_ctx) acc[0] = acc[1] = -INFINITY;
+      if (page * DD_T + gl + 8 >= n_ctx) acc[2] = acc[3] = -INFINITY;
+    }
+    // ---- running soft-max per column
+    float alpha[2], pr[4];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      float pm = fmaxf(acc[c], acc[2 + c]);
+      pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 4));
+      pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 8));
+      pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 16));
+      const float mn = fmaxf(m_run[c], pm);
+      if (mn == -INFINITY) {
+        alpha[c] = 1.f; pr[c] = 0.f; pr[2 + c] = 0.f;
+      } else {
+        alpha[c] = exp2f(m_run[c] - mn);
+        pr[c] = exp2f(acc[c] - mn);
+        pr[2 + c] = exp2f(acc[2 + c] - mn);
+      }
+      l_run[c] = l_run[c] * alpha[c] + pr[c] + pr[2 + c];
+      m_run[c] = mn;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      o[i][0] *= alpha[0]; o[i][1] *= alpha[1]; o[i][2] *= alpha[0]; o[i][3] *= alpha[1];
+    }
+    // ---- P^T as the B operand: tokens {2t, 2t+1} and {2t+8, 2t+9} of column gl
+    const uint32_t pb0 = dd_movmatrix_trans(dd_pack_bf16(pr[0], pr[1]));
+    const uint32_t pb1 = dd_movmatrix_trans(dd_pack_bf16(pr[2], pr[3]));
+    // ---- O^T += V^T P^T; MMA tile i has rows gl -> channel 8gl+i and gl+8 -> channel 64+8gl+i
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int w = i >> 1;
+      const uint32_t sel = (i & 1) ? 0x7632u : 0x5410u;
+      const uint32_t a0 = __byte_perm(v[0][0][w], v[1][0][w], sel);
+      const uint32_t a1 = __byte_perm(v[0][1][w], v[1][1][w], sel);
+      const uint32_t a2 = __byte_perm(v[2][0][w], v[3][0][w], sel);
+      const uint32_t a3 = __byte_perm(v[2][1][w], v[3][1][w], sel);
+      dd_mma_bf16(o[i], a0, a1, a2, a3, pb0, pb1);
+    }
+  }
+  // l over the 8 row groups of the warp
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 4);
+    l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 8);
+    l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 16);
+  }
+  // ---- merge the warps of the block
+  if (gl == 0) {
+    sm_ml[warp][2 * t] = make_float2(m_run[0], l_run[0]);
+    sm_ml[warp][2 * t + 1] = make_float2(m_run[1], l_run[1]);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    sm_o[warp][2 * t][8 * gl + i] = o[i][0];
+    sm_o[warp][2 * t + 1][8 * gl + i] = o[i][1];
+    sm_o[warp][2 * t][64 + 8 * gl + i] = o[i][2];
+    sm_o[warp][2 * t + 1][64 + 8 * gl + i] = o[i][3];
+  }
+  __syncthreads();
+  if (threadIdx.x < ATTN_ROWS) {
+    const int n = threadIdx.x;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < ATTN_WARPS; ++w) M = fmaxf(M, sm_ml[w][n].x);
+    float L = 0.f;
+#pragma unroll
+    for (int w = 0; w < ATTN_WARPS; ++w) {
+      const float sc = (M == -INFINITY) ? 0.f : exp2f(sm_ml[w][n].x - M);
+      sm_scale[w][n] = sc;
+      L += sm_ml[w][n].y * sc;
+    }
+    sm_ml[0][n] = make_float2(M, L);             // block result, read after the next barrier
+  }
+  __syncthreads();
+  const int d = threadIdx.x;                     // one channel per thread, all rows
+  float ob[ATTN_ROWS];
+#pragma unroll
+  for (int n = 0; n < ATTN_ROWS; ++n) {
+    float a = 0.f;
+#pragma unroll
+    for (int w = 0; w < ATTN_WARPS; ++w) a += sm_o[w][n][d] * sm_scale[w][n];
+    ob[n] = a;
+  }
+
+  if (n_splits == 1) {
+#pragma unroll
+    for (int n = 0; n < ATTN_ROWS; ++n) {
+      if (n < n_rows) {
+        const int tq = n / G, hh = n - tq * G;
+        const float2 ml = sm_ml[0][n];
+        const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+        out[row * DD_D + d] = __float2bfloat16_rn(ml.y > 0.f ? ob[n] / ml.y : 0.f);
+        if (out_lse && d == 0) out_lse[row] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
+      }
+    }
+    return;
+  }
+
+  // ---- several splits: publish the partial, the last block to arrive merges
+  {
+    float* po = part_o + ((bg * n_splits + split) * ATTN_ROWS) * DD_D;
+#pragma unroll
+    for (int n = 0; n < ATTN_ROWS; ++n) po[n * DD_D + d] = ob[n];
+    if (d < ATTN_ROWS) part_ml[(bg * n_splits + split) * ATTN_ROWS + d] = sm_ml[0][d];
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned prev = atomicAdd(&ticket[bg], 1u);
+    sm_last = (prev == (unsigned)(n_splits - 1));
+  }
+  __syncthreads();
+  if (!sm_last) return;
+  __threadfence();
+  if (threadIdx.x == 0) ticket[bg] = 0u;         // ready for the next launch
+#pragma unroll 1
+  for (int n = 0; n < n_rows; ++n) {
+    const float2* pml = part_ml + bg * n_splits * ATTN_ROWS + n;
+    float M = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, __ldcg(&pml[s * ATTN_ROWS].x));
+    float L = 0.f, a = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+      const float ms = __ldcg(&pml[s * ATTN_ROWS].x);
+      const float sc = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
+      L += __ldcg(&pml[s * ATTN_ROWS].y) * sc;
+      a += __ldcg(part_o + ((bg * n_splits + s) * ATTN_ROWS + n) * DD_D + d) * sc;
+    }
+    const int tq = n / G, hh = n - tq * G;
+    const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+    out[row * DD_D + d] = __float2bfloat16_rn(L > 0.f ? a / L : 0.f);
+    if (out_lse && d == 0) out_lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+  }
+}
+
+int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
+                   float* out_lse, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const int S = ctx->attn_splits;
+  const int pps = (c.k_pages + S - 1) / S;
+  dim3 grid(S, c.n_kv_heads, c.batch);
+  dd_attn_kernel<<<grid, ATTN_THREADS, 0, st>>>((const __nv_bfloat16*)q, slot, idx, ctx_len, (__nv_bfloat16*)out,
+                                                out_lse, ctx->attn_part_o, ctx->attn_part_ml, ctx->attn_ticket,
+                                                c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, S, pps);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}

@@ -1,0 +1,359 @@
+// Landmark build (set-up), page scoring and per-KV-head top-k selection.
+//
+// Scoring streams the landmarks of a layer once from HBM: the 16 landmarks of a tile are the M rows
+// of a warp-level bf16 MMA, the G query heads that share the KV head are its N columns. The top-k
+// kernel turns the per-head logits into log-probabilities with the per-head log-sum-exp, takes the
+// group maximum, and finds the k-th largest by an MSB-first radix select on order-preserving keys,
+// followed by an ordered compaction that emits ascending page numbers.
+#include "dd_common.cuh"
+
+// ------------------------------------------------------------------------------------------------
+// Landmarks: mean of the valid keys of a page, fp32 sum in token order, fp32 divide, RNE to bf16.
+// One warp per page; a lane owns 4 consecutive channels.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) dd_landmark_kernel(const __nv_bfloat16* __restrict__ kv,
+                                                          const int* __restrict__ ctx_len,
+                                                          __nv_bfloat16* __restrict__ lm, int Hkv, int P,
+                                                          long long n_pages_total) {
+  const int lane = threadIdx.x & 31;
+  long long page = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long stride = (long long)gridDim.x * (blockDim.x >> 5);
+  for (; page < n_pages_total; page += stride) {
+    const int p = (int)(page % P);
+    const int b = (int)(page / ((long long)P * Hkv));
+    int cnt = ctx_len[b] - p * DD_T;
+    cnt = cnt > DD_T ? DD_T : cnt;
+    const __nv_bfloat16* src = kv + page * (2 * DD_T * DD_D) + lane * 4;   // K half comes first
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int i = 0; i < cnt; ++i) {
+      uint2 w = *reinterpret_cast<const uint2*>(src + i * DD_D);
+      __nv_bfloat162 lo = *reinterpret_cast<__nv_bfloat162*>(&w.x);
+      __nv_bfloat162 hi = *reinterpret_cast<__nv_bfloat162*>(&w.y);
+      a0 = __fadd_rn(a0, __low2float(lo));
+      a1 = __fadd_rn(a1, __high2float(lo));
+      a2 = __fadd_rn(a2, __low2float(hi));
+      a3 = __fadd_rn(a3, __high2float(hi));
+    }
+    uint2 o = make_uint2(0u, 0u);
+    if (cnt > 0) {
+      const float c = (float)cnt;
+      __nv_bfloat162 lo = __floats2bfloat162_rn(__fdiv_rn(a0, c), __fdiv_rn(a1, c));
+      __nv_bfloat162 hi = __floats2bfloat162_rn(__fdiv_rn(a2, c), __fdiv_rn(a3, c));
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+    }
+    *reinterpret_cast<uint2*>(lm + page * DD_D + lane * 4) = o;
+  }
+}
+
+int dd_launch_build_landmarks(dd_ctx* ctx, const void* kv_dev, const int* ctx_len, void* landmarks, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const long long total = (long long)c.batch * c.n_kv_heads * c.max_pages;
+  const int warps_per_block = 8;
+  long long blocks = (total + warps_per_block - 1) / warps_per_block;
+  const long long cap = (long long)ctx->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  dd_landmark_kernel<<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(
+      (const __nv_bfloat16*)kv_dev, ctx_len, (__nv_bfloat16*)landmarks, c.n_kv_heads, c.max_pages, total);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scoring. Grid (tile, KV head, request); 4 warps; each warp scores two 16-page MMA tiles.
+//
+// Fragment trick: the dot product does not care in which order the 128 channels are summed, so a
+// thread feeds the MMA's k-slots {2t, 2t+1, 2t+8, 2t+9} of two consecutive k-steps with the eight
+// consecutive channels [32*kk + 8t, 32*kk + 8t + 8) of its row — one 16-byte load — and the query
+// fragment uses the same assignment. The four threads of a row then read 64 contiguous bytes.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) dd_score_kernel(const __nv_bfloat16* __restrict__ q, int q_req_stride,
+                                                       int q_token_off, const __nv_bfloat16* __restrict__ lm,
+                                                       const int* __restrict__ n_pages, float* __restrict__ s_out,
+                                                       float2* __restrict__ part, int P, int G, int Hkv,
+                                                       int n_tiles) {
+  const int tile = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const int Hq = Hkv * G;
+  int np = n_pages[b];
+  np = np > P ? P : np;
+  const int p_base = tile * DD_SCORE_TILE;
+
+  __shared__ float2 red[4][8];
+
+  float m_run[2] = {-INFINITY, -INFINITY};   // heads 2t, 2t+1
+  float l_run[2] = {0.f, 0.f};
+
+  if (p_base < np) {
+    // query fragments: column n = gl is head g*G + gl
+    uint4 qf[4];
+    if (gl < G) {
+      const uint4* qrow = reinterpret_cast<const uint4*>(q + (size_t)b * q_req_stride + q_token_off +
+                                                         (size_t)(g * G + gl) * DD_D);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = __ldg(qrow + kk * 4 + t);
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const __nv_bfloat16* lm_bg = lm + (size_t)(b * Hkv + g) * P * DD_D;
+    uint4 lo[2][4], hi[2][4];
+    int prow[2][2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      const int p0 = p_base + (warp * 2 + mt) * 16;
+      prow[mt][0] = p0 + gl;
+      prow[mt][1] = p0 + gl + 8;
+      const int pa = prow[mt][0] < P ? prow[mt][0] : P - 1;   // stay inside the tensor; result discarded
+      const int pb = prow[mt][1] < P ? prow[mt][1] : P - 1;
+      const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D);
+      const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        lo[mt][kk] = dd_ld_stream(ra + kk * 4 + t);
+        hi[mt][kk] = dd_ld_stream(rb + kk * 4 + t);
+      }
+    }
+    const float scale = rsqrtf((float)DD_D);
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        dd_mma_bf16(acc, lo[mt][kk].x, hi[mt][kk].x, lo[mt][kk].y, hi[mt][kk].y, qf[kk].x, qf[kk].y);
+        dd_mma_bf16(acc, lo[mt][kk].z, hi[mt][kk].z, lo[mt][kk].w, hi[mt][kk].w, qf[kk].z, qf[kk].w);
+      }
+      // acc[0], acc[1]: page prow[mt][0], heads 2t, 2t+1; acc[2], acc[3]: page prow[mt][1]
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int p = prow[mt][r];
+        if (p < np) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            const int h = 2 * t + c;
+            if (h < G) {
+              const float v = acc[2 * r + c] * scale;
+              s_out[((size_t)(b * Hkv + g) * P + p) * G + h] = v;
+              const float mn = fmaxf(m_run[c], v);
+              l_run[c] = l_run[c] * expf(m_run[c] - mn) + expf(v - mn);
+              m_run[c] = mn;
+            }
+          }
+        }
+      }
+    }
+  }
+  // reduce (m, l) over the 8 row groups of the warp, then over the 4 warps
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m_run[c], off);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l_run[c], off);
+      dd_ml_merge(m_run[c], l_run[c], m2, l2, false);
+    }
+  }
+  if (gl == 0) {
+    red[warp][2 * t] = make_float2(m_run[0], l_run[0]);
+    red[warp][2 * t + 1] = make_float2(m_run[1], l_run[1]);
+  }
+  __syncthreads();
+  if (threadIdx.x < G) {
+    float m = red[0][threadIdx.x].x, l = red[0][threadIdx.x].y;
+#pragma unroll
+    for (int w = 1; w < 4; ++w) dd_ml_merge(m, l, red[w][threadIdx.x].x, red[w][threadIdx.x].y, false);
+    part[((size_t)b * Hq + g * G + threadIdx.x) * n_tiles + tile] = make_float2(m, l);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Top-k of one (request, KV head) per thread block.
+// ------------------------------------------------------------------------------------------------
+constexpr int TOPK_THREADS = 1024;
+constexpr int TOPK_SMEM_KEYS = 16384;          // requests up to this many pages keep their keys in shared memory
+constexpr int RADIX_BITS = 11;
+constexpr int RADIX_BINS = 1 << RADIX_BITS;
+
+// fp32 -> uint32 with the same order
+__device__ __forceinline__ uint32_t dd_orderable(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive prefix sum over the 1024 threads of the block; `total` is returned to every thread.
+__device__ __forceinline__ unsigned dd_block_scan_excl(unsigned v, unsigned* warp_tot, unsigned& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned inc = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, inc, off);
+    if (lane >= off) inc += n;
+  }
+  __syncthreads();                               // warp_tot may still be read from the previous scan
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  unsigned wt = warp_tot[lane];                  // 32 warps
+  unsigned winc = wt;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, winc, off);
+    if (lane >= off) winc += n;
+  }
+  total = __shfl_sync(0xffffffffu, winc, 31);
+  const unsigned wexcl = __shfl_sync(0xffffffffu, winc - wt, warp);
+  return wexcl + inc - v;
+}
+
+__global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
+    const float* __restrict__ s, const float2* __restrict__ part, const int* __restrict__ n_pages,
+    uint32_t* __restrict__ gkeys, int* __restrict__ out_idx, float* __restrict__ out_scores, int P, int G, int Hkv,
+    int n_tiles, int k, int forced, int* err_word) {
+  extern __shared__ uint32_t smem_keys[];
+  __shared__ unsigned hist[RADIX_BINS];
+  __shared__ unsigned warp_tot[32];
+  __shared__ float lse_s[8];
+  __shared__ unsigned sh_min, sh_max, sh_bin, sh_above;
+
+  const int g = blockIdx.x, b = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Hq = Hkv * G;
+  const size_t bg = (size_t)b * Hkv + g;
+  int np = n_pages[b];
+  if (np > P || np < k) {
+    if (tid == 0) dd_report(err_word, DD_ERR_INDEX_RANGE, np);
+    np = np > P ? P : (np < 0 ? 0 : np);
+  }
+  const int k_eff = k < np ? k : np;
+  const int forced_eff = forced < k_eff ? forced : k_eff;
+  const int n_free = np - forced_eff;            // pages [n_free, np) are forced
+  const int k_free = k_eff - forced_eff;
+  int* out = out_idx + bg * k;
+  if (tid == 0) { sh_min = 0xFFFFFFFFu; sh_max = 0u; }
+
+  // 1. log-sum-exp of every head of the group from the per-tile partials
+  if (warp < G) {
+    const int tiles = (np + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
+    const float2* pp = part + ((size_t)b * Hq + g * G + warp) * n_tiles;
+    float m = -INFINITY, l = 0.f;
+    for (int i = lane; i < tiles; i += 32) {
+      const float2 v = pp[i];
+      dd_ml_merge(m, l, v.x, v.y, false);
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l, off);
+      dd_ml_merge(m, l, m2, l2, false);
+    }
+    if (lane == 0) lse_s[warp] = m + logf(l);
+  }
+  __syncthreads();
+
+  // 2. keys: group maximum of the log-probabilities, order-preserving integer form
+  uint32_t* keys = (np <= TOPK_SMEM_KEYS) ? smem_keys : gkeys + bg * P;
+  {
+    float lse[8];
+#pragma unroll
+    for (int h = 0; h < 8; ++h) lse[h] = h < G ? lse_s[h] : 0.f;
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+    const float* sp = s + bg * (size_t)P * G;
+    for (int p = tid; p < np; p += TOPK_THREADS) {
+      float c = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < 8; ++h)
+        if (h < G) c = fmaxf(c, sp[(size_t)p * G + h] - lse[h]);
+      if (out_scores) out_scores[bg * P + p] = expf(c);
+      uint32_t key = dd_orderable(c);
+      if (p >= n_free) key = 0xFFFFFFFFu;
+      else { kmin = min(kmin, key); kmax = max(kmax, key); }
+      keys[p] = key;
+    }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { atomicMin(&sh_min, kmin); atomicMax(&sh_max, kmax); }
+  }
+  __syncthreads();
+
+  // 3. radix select of the k_free-th largest key among the non-forced pages
+  uint32_t thr = 0xFFFFFFFFu;
+  unsigned k_rem = 0;
+  if (k_free > 0) {
+    const uint32_t kmin = sh_min;
+    const uint32_t range = sh_max - kmin;
+    const int nbits = 32 - __clz(range);
+    const int passes = (nbits + RADIX_BITS - 1) / RADIX_BITS;
+    unsigned long long prefix = 0;
+    k_rem = (unsigned)k_free;
+    for (int pass = 0; pass < passes; ++pass) {
+      const int shift = (passes - 1 - pass) * RADIX_BITS;
+      for (int i = tid; i < RADIX_BINS; i += TOPK_THREADS) hist[i] = 0u;
+      __syncthreads();
+      for (int p = tid; p < n_free; p += TOPK_THREADS) {
+        const unsigned long long rel = (unsigned long long)(keys[p] - kmin);
+        if ((rel >> (shift + RADIX_BITS)) == prefix) atomicAdd(&hist[(unsigned)(rel >> shift) & (RADIX_BINS - 1)], 1u);
+      }
+      __syncthreads();
+      // thread i owns bins 2047-2i and 2046-2i; scan from the top bin downwards
+      const unsigned h_hi = hist[RADIX_BINS - 1 - 2 * tid], h_lo = hist[RADIX_BINS - 2 - 2 * tid];
+      unsigned total;
+      const unsigned above = dd_block_scan_excl(h_hi + h_lo, warp_tot, total);
+      if (above < k_rem && k_rem <= above + h_hi + h_lo) {
+        if (above + h_hi >= k_rem) { sh_bin = RADIX_BINS - 1 - 2 * tid; sh_above = above; }
+        else { sh_bin = RADIX_BINS - 2 - 2 * tid; sh_above = above + h_hi; }
+      }
+      __syncthreads();
+      prefix = (prefix << RADIX_BITS) | sh_bin;
+      k_rem -= sh_above;
+      __syncthreads();
+    }
+    thr = kmin + (uint32_t)prefix;               // k_rem of the keys equal to thr are still to be taken
+  }
+
+  // 4. ordered compaction: ascending page numbers; equal keys are taken from the lowest page up
+  unsigned base_gt = 0, base_eq = 0;
+  for (int c0 = 0; c0 < np; c0 += TOPK_THREADS) {
+    const int p = c0 + tid;
+    unsigned gt = 0, eq = 0;
+    if (p < np) {
+      const uint32_t key = keys[p];
+      if (p >= n_free || key > thr) gt = 1;
+      else if (key == thr) eq = 1;
+    }
+    unsigned total;
+    const unsigned ex = dd_block_scan_excl(gt | (eq << 16), warp_tot, total);
+    const unsigned eq_before = base_eq + (ex >> 16);
+    if (gt || (eq && eq_before < k_rem)) {
+      const unsigned pos = base_gt + (ex & 0xFFFFu) + min(eq_before, k_rem);
+      if (pos < (unsigned)k) out[pos] = p;
+    }
+    base_gt += total & 0xFFFFu;
+    base_eq += total >> 16;
+  }
+  // precondition k <= n_pages violated: pad with the last valid page so that later stages stay in range
+  for (int j = k_eff + tid; j < k; j += TOPK_THREADS) out[j] = np > 0 ? np - 1 : 0;
+}
+
+int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
+                     const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const int G = ctx->G;
+  dim3 sgrid(ctx->score_tiles, c.n_kv_heads, c.batch);
+  dd_score_kernel<<<sgrid, 128, 0, st>>>((const __nv_bfloat16*)q, q_tokens_in_tensor * c.n_q_heads * DD_D,
+                                         q_token * c.n_q_heads * DD_D, (const __nv_bfloat16*)landmarks, n_pages,
+                                         ctx->score_s, ctx->score_part, c.max_pages, G, c.n_kv_heads,
+                                         ctx->score_tiles);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  dim3 tgrid(c.n_kv_heads, c.batch);
+  dd_topk_kernel<<<tgrid, TOPK_THREADS, TOPK_SMEM_KEYS * sizeof(uint32_t), st>>>(
+      ctx->score_s, ctx->score_part, n_pages, ctx->topk_keys, out_idx, out_scores, c.max_pages, G, c.n_kv_heads,
+      ctx->score_tiles, c.k_pages, c.forced_recent_pages, ctx->err_word);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}
+
+int dd_select_setup(dd_ctx* ctx) {
+  DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(TOPK_SMEM_KEYS * sizeof(uint32_t))));
+  return DD_OK;
+}

@@ -1,0 +1,197 @@
+"""GPU parity of the pipelined layer step (ring + events) against the oracle's multi-step chain,
+its invariance to ring depth and gather engine, its call-order checks, and a sampled check at
+config 2's full launch configuration (32 layers, batch 8, 2048 pages, 128 selected)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dd_oracle as orc
+from paper_2607_26475_b200 import workloads as wl
+from tests._util import check_attention, check_selection, f32, raw16
+
+pytestmark = pytest.mark.gpu
+
+HQ, HKV, D, T = 32, 8, 128, 16
+
+
+@pytest.fixture(scope="module")
+def dd():
+    from paper_2607_26475_b200 import binding
+    return binding
+
+
+def _inputs(w, S, ragged=True):
+    L, B = w.n_layers, w.batch
+    store = [torch.stack([wl.kv_slab(w, l, b) for b in range(B)]).pin_memory() for l in range(L)]
+    ctx_len = wl.ctx_lens(w, ragged=ragged)
+    npg = ((ctx_len + T - 1) // T).to(torch.int32)
+    lms = [torch.from_numpy(orc.build_landmarks(f32(store[l][:, :, :, 0]), ctx_len.numpy())).to(torch.bfloat16)
+           for l in range(L)]
+    q_init = torch.stack([wl.queries(w, -1, l)[:, 1] for l in range(L)])                   # [L, B, Hq, d]
+    q_steps = torch.stack([torch.stack([wl.queries(w, t, l) for l in range(L)]) for t in range(S)])
+    return store, lms, ctx_len, npg, q_init, q_steps
+
+
+def _run(dd, w, S, inp, depth, mode=0, read_idx=True):
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    L, B = w.n_layers, w.batch
+    c = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
+                   forced_recent_pages=w.forced_recent_pages, ring_depth=depth, gather_mode=mode)
+    lm_dev = [x.cuda() for x in lms]
+    c.bind(lm_dev, store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qd = q_steps.cuda()
+    outs = torch.zeros_like(qd)
+    idxs = []
+    for t in range(S):
+        if read_idx:
+            idxs.append(torch.stack([c.get_indices(t & 1, l) for l in range(L)]).cpu().numpy())
+        for l in range(L):
+            c.decode_layer_step(t, l, qd[t, l], outs[t, l])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    c.close()
+    return outs, (np.stack(idxs) if read_idx else None)
+
+
+def test_chain_matches_oracle_and_is_invariant_to_ring_depth_and_engine(dd):
+    S = 3
+    w = wl.small(wl.CONFIGS[4], n_layers=3, batch=2, ctx=16 * 90, budget=16 * 12, recent_window=32)
+    inp = _inputs(w, S)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    outs, idxs = _run(dd, w, S, inp, depth=2)
+    # selection of every (step, layer): band rule against the oracle's scores for the query that produced it
+    for t in range(S):
+        for l in range(w.n_layers):
+            qsel = f32(q_init[l]) if t == 0 else f32(q_steps[t - 1, l][:, 1])
+            _, sc = orc.select_topk(qsel, f32(lms[l]), npg.numpy(), w.k_pages, w.forced_recent_pages)
+            for b in range(w.batch):
+                for h in range(HKV):
+                    check_selection(idxs[t, l, b, h], sc[b][h], w.k_pages, w.forced_recent_pages)
+            # attention over the GPU's own set
+            slot = orc.gather_kv(f32(store[l]), idxs[t, l])
+            want, _ = orc.sparse_decode_attn(f32(q_steps[t, l]), slot, idxs[t, l], ctx_len.numpy(), T)
+            check_attention(outs[t, l], want)
+    # the whole chain in the oracle, when every set matched exactly
+    o_outs, o_idxs = orc.decode_chain(f32(q_init), f32(q_steps), [f32(x) for x in lms], [f32(x) for x in store],
+                                      npg.numpy(), ctx_len.numpy(), w.k_pages, T, w.forced_recent_pages)
+    if np.array_equal(o_idxs[:S], idxs):
+        check_attention(outs, o_outs)
+    # same bits whatever the ring depth, the gather engine, and with no host reads in between
+    for depth, mode, read in [(3, 0, True), (4, 0, False), (2, 1, False), (2, 0, False)]:
+        o2, i2 = _run(dd, w, S, inp, depth=depth, mode=mode, read_idx=read)
+        assert np.array_equal(raw16(o2), raw16(outs)), (depth, mode)
+        if read:
+            assert np.array_equal(i2, idxs)
+
+
+def test_single_layer_model_with_a_deeper_ring(dd):
+    """Config 1's shape: one layer, two slots; the next step's gather is released by this step's selection."""
+    S = 4
+    w = wl.small(wl.CONFIGS[1], steps=S)
+    inp = _inputs(w, S, ragged=False)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    outs, idxs = _run(dd, w, S, inp, depth=2)
+    for t in range(S):
+        slot = orc.gather_kv(f32(store[0]), idxs[t, 0])
+        want, _ = orc.sparse_decode_attn(f32(q_steps[t, 0]), slot, idxs[t, 0], ctx_len.numpy(), T)
+        check_attention(outs[t, 0], want)
+        qsel = f32(q_init[0]) if t == 0 else f32(q_steps[t - 1, 0][:, 1])
+        _, sc = orc.select_topk(qsel, f32(lms[0]), npg.numpy(), w.k_pages)
+        for h in range(HKV):
+            check_selection(idxs[t, 0, 0, h], sc[0][h], w.k_pages, 0)
+
+
+def test_call_order_is_checked(dd):
+    w = wl.small(wl.CONFIGS[2], n_layers=2, batch=1, ctx=16 * 40, budget=16 * 4)
+    inp = _inputs(w, 1, ragged=False)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    c = dd.Context(n_layers=2, batch=1, max_pages=40, k_pages=4)
+    q = q_steps[0, 0].cuda()
+    out = torch.empty_like(q)
+    with pytest.raises(dd.DDError) as e:
+        c.prime(q_init.cuda())
+    assert e.value.code == dd.DD_ERR_STATE
+    with pytest.raises(dd.DDError) as e:
+        c.decode_layer_step(0, 0, q, out)
+    assert e.value.code == dd.DD_ERR_STATE
+    with pytest.raises(dd.DDError) as e:
+        c.bind([x.cuda() for x in lms], [s.clone() for s in store], npg.cuda(), ctx_len.cuda())   # not pinned
+    assert e.value.code == dd.DD_ERR_NOT_PINNED
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    with pytest.raises(dd.DDError) as e:
+        c.decode_layer_step(0, 1, q, out)          # layer 0 comes first
+    assert e.value.code == dd.DD_ERR_STATE
+    c.decode_layer_step(0, 0, q, out)
+    c.decode_layer_step(0, 1, q, out)
+    with pytest.raises(dd.DDError) as e:
+        c.decode_layer_step(0, 1, q, out)          # already done
+    assert e.value.code == dd.DD_ERR_STATE
+    c.decode_layer_step(1, 0, q, out)
+    c.sync()
+    assert c.device_error() == (0, 0)
+    c.close()
+
+
+def test_invalid_configurations_are_rejected(dd):
+    for kw in (dict(head_dim=64), dict(page_tokens=32), dict(k_pages=50), dict(ring_depth=1), dict(n_q_heads=30),
+               dict(forced_recent_pages=9), dict(n_q_heads=64, n_q_tokens=2), dict(gather_mode=5)):
+        args = dict(n_layers=1, batch=1, max_pages=40, k_pages=8)
+        args.update(kw)
+        with pytest.raises(dd.DDError) as e:
+            dd.Context(**args)
+        assert e.value.code == dd.DD_ERR_INVALID_ARG
+
+
+def test_config2_launch_configuration_sampled(dd):
+    """Config 2 as the benchmark launches it (L=32, B=8, 32768-token contexts, 2048 of them selected per KV
+    head, ring depth 2). The host store aliases two physical layers to stay small; sampled (step, layer,
+    request) outputs are checked one by one against the oracle."""
+    w = wl.CONFIGS[2]
+    L, B, P, k, S, n_phys = w.n_layers, w.batch, w.n_pages, w.k_pages, 2, 2
+    ctx_len = wl.ctx_lens(w)
+    npg = torch.full((B,), P, dtype=torch.int32)
+    c = dd.Context(n_layers=L, batch=B, max_pages=P, k_pages=k)
+    phys, lms = [], []
+    for l in range(n_phys):
+        dev = torch.stack([wl.kv_slab(w, l, b, device="cuda") for b in range(B)])
+        lm = torch.empty((B, HKV, P, D), dtype=torch.bfloat16, device="cuda")
+        c.build_landmarks(dev, ctx_len.cuda(), lm)
+        host = torch.empty(dev.shape, dtype=torch.bfloat16, pin_memory=True)
+        host.copy_(dev)
+        phys.append(host)
+        lms.append(lm)
+        del dev
+    torch.cuda.synchronize()
+    store = [phys[l % n_phys] for l in range(L)]
+    lm_l = [lms[l % n_phys] for l in range(L)]
+    q_init = torch.stack([wl.queries(w, -1, l)[:, 1] for l in range(L)])
+    q_steps = torch.stack([torch.stack([wl.queries(w, t, l) for l in range(L)]) for t in range(S)])
+    c.bind(lm_l, store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qd = q_steps.cuda()
+    outs = torch.zeros_like(qd)
+    idxs = []
+    for t in range(S):
+        idxs.append(torch.stack([c.get_indices(t & 1, l) for l in range(L)]).cpu().numpy())
+        for l in range(L):
+            c.decode_layer_step(t, l, qd[t, l], outs[t, l])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    n_exact = n_all = 0
+    for t, l, b in [(0, 0, 0), (0, 17, 7), (1, 31, 3), (1, 16, 0)]:
+        kv_b = f32(store[l][b:b + 1])
+        lm_want = orc.build_landmarks(kv_b[:, :, :, 0], ctx_len[b:b + 1].numpy())
+        assert np.array_equal(f32(lm_l[l][b:b + 1]), lm_want), "device-built landmarks differ from the oracle's"
+        qsel = f32(q_init[l][b:b + 1]) if t == 0 else f32(q_steps[t - 1, l][b:b + 1, 1])
+        _, sc = orc.select_topk(qsel, lm_want, npg[b:b + 1].numpy(), k)
+        got = idxs[t][l][b:b + 1]
+        for h in range(HKV):
+            n_exact += check_selection(got[0, h], sc[0][h], k, 0)
+            n_all += 1
+        slot = orc.gather_kv(kv_b, got)
+        want, _ = orc.sparse_decode_attn(f32(q_steps[t, l][b:b + 1]), slot, got, ctx_len[b:b + 1].numpy(), T)
+        check_attention(outs[t, l][b:b + 1], want)
+    print(f"exact index sets: {n_exact}/{n_all}")
+    c.close()
