@@ -92,6 +92,21 @@ def _ptr(t):
     return t.data_ptr()
 
 
+class _DevMem:
+    """Raw device memory as a CUDA-array-interface object, so that torch can view it."""
+
+    def __init__(self, ptr: int, shape, typestr: str):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False),
+                                         "version": 2, "strides": None}
+
+
+def _view(ptr: int, shape, kind: str) -> torch.Tensor:
+    """Zero-copy torch view of library-owned device memory (kind: 'i4' or 'bf16')."""
+    if kind == "bf16":
+        return torch.as_tensor(_DevMem(ptr, shape, "<i2"), device="cuda").view(torch.bfloat16)
+    return torch.as_tensor(_DevMem(ptr, shape, "<" + kind), device="cuda")
+
+
 def _stream(s) -> int:
     if s is None:
         return torch.cuda.current_stream().cuda_stream
@@ -157,12 +172,8 @@ class Context:
         """A copy of ring slot `slot` as [B, Hkv, 2, k*T, d] bf16 (synchronises; for tests)."""
         c = self.cfg
         shape = (c.batch, c.n_kv_heads, 2, c.k_pages * c.page_tokens, c.head_dim)
-        out = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
         torch.cuda.synchronize()
-        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), self.slot_ptr(slot), self.slot_bytes(), 3)
-        if int(rc) != 0:
-            raise RuntimeError(f"cudaMemcpy failed: {rc}")
-        return out
+        return _view(self.slot_ptr(slot), shape, "bf16").clone()
 
     def sync(self, timeout_s: float = 60.0):
         self._check(lib.dd_sync(self._h, timeout_s))
@@ -207,9 +218,5 @@ class Context:
         p = C.c_void_p()
         self._check(lib.dd_get_indices(self._h, step_parity, layer, C.byref(p)))
         c = self.cfg
-        out = torch.empty((c.batch, c.n_kv_heads, c.k_pages), dtype=torch.int32, device="cuda")
         torch.cuda.synchronize()
-        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p.value, out.numel() * 4, 3)
-        if int(rc) != 0:
-            raise RuntimeError(f"cudaMemcpy failed: {rc}")
-        return out
+        return _view(p.value, (c.batch, c.n_kv_heads, c.k_pages), "i4").clone()
