@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse decode hot path: decode tokens/s on synthetic Llama-3-8B-shaped workloads.
+
+A "step" is one decode step of the whole path: for each of the L layers, attention over the set gathered
+for it, the selection of the next step's set from the speculated token, and the host->HBM gather of a
+later layer on the side stream (dd_decode_layer_step). `value` counts output tokens only (B per step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange step.
+`--impl reference` times the CPU oracle on the host cores instead (a deliberately slow program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tok/s"
+
+
+def log(msg):
+    print(f"[bench] {msg}", file=sys.stderr, flush=True)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="workload number (2 = batch 8, 32K context, budget 2048)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--phys-layers", type=int, default=0, help="distinct layers kept in the host store (0 = as many as fit)")
+    ap.add_argument("--ring-depth", type=int, default=2)
+    ap.add_argument("--gather-mode", default="loads", choices=["loads", "bulk"])
+    ap.add_argument("--gather-ctas", type=int, default=0)
+    ap.add_argument("--attn-splits", type=int, default=0)
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling of small cases only)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of small cases only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stages", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(index)], stdout=subprocess.PIPE, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(w, n_layers_cap=4, min_seconds=8.0):
+    """Times the oracle, as it stands, on whole layers of the workload (all requests, one step):
+    selection from the speculated token, page gather, attention of both tokens. Returns tok/s scaled to
+    a full step of w.n_layers layers."""
+    import numpy as np
+    from oracle import dd_oracle as orc
+    from paper_2607_26475_b200 import workloads as wl
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    ctx_len = wl.ctx_lens(w).numpy()
+    npg = (ctx_len + w.page_tokens - 1) // w.page_tokens
+    layers, t_total = 0, 0.0
+    split = {"select": 0.0, "gather": 0.0, "attn": 0.0}
+    while layers < n_layers_cap and (layers == 0 or t_total < min_seconds):
+        l = layers
+        import torch
+        kv = torch.stack([wl.kv_slab(w, l, b) for b in range(w.batch)])
+        kv32 = kv.float().numpy()
+        lm = orc.build_landmarks(kv32[:, :, :, 0], ctx_len)             # set-up, not timed
+        q = wl.queries(w, 0, l).float().numpy()
+        t0 = time.perf_counter()
+        idx, _ = orc.select_topk(q[:, 1], lm, npg, w.k_pages, w.forced_recent_pages)
+        t1 = time.perf_counter()
+        slot = orc.gather_kv(kv32, idx)
+        t2 = time.perf_counter()
+        orc.sparse_decode_attn(q, slot, idx, ctx_len, w.page_tokens)
+        t3 = time.perf_counter()
+        split["select"] += t1 - t0
+        split["gather"] += t2 - t1
+        split["attn"] += t3 - t2
+        t_total += t3 - t0
+        layers += 1
+        del kv, kv32, slot
+    per_layer = t_total / layers
+    value = w.batch / (per_layer * w.n_layers)
+    return {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{layers} layer(s) x all {w.batch} requests x 1 step of {w.name}, scaled to {w.n_layers} layers",
+            "us_per_layer": {k: v / layers * 1e6 for k, v in split.items()}, "seconds": t_total}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_26475_b200 import workloads as wl
+    w = wl.CONFIGS[args.config]
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, n_layers_cap=1, min_seconds=0.0)
+    vals, info = [], None
+    t0 = time.time()
+    for _ in range(args.steps):
+        info = oracle_sample(w, n_layers_cap=1, min_seconds=0.0)
+        vals.append(info["value"])
+        if time.time() - t0 > 150:
+            break
+    value = len(vals) / sum(1.0 / v for v in vals)
+    ms = w.batch / value * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": len(vals), "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.batch, "ctx": w.ctx, "budget": w.budget, "layers": w.n_layers},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": info["cores"], "kind": "oracle",
+                             "sample": "each step = 1 layer x all requests, scaled to a full step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    import torch.distributed as dist
+    from paper_2607_26475_b200 import binding as dd
+    from paper_2607_26475_b200 import workloads as wl
+    from paper_2607_26475_b200.store import HostStore, available_host_bytes
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    w = wl.CONFIGS[args.config]
+    if args.layers or args.batch:
+        w = wl.small(w, n_layers=args.layers or w.n_layers, batch=args.batch or w.batch)
+    L, B, K, W = w.n_layers, w.batch, args.steps, max(args.warmup, 0)
+    hbm_peak, peak_src = measured_peaks()
+
+    compute = torch.cuda.Stream()
+    copy = torch.cuda.Stream(priority=0)
+    gm = dd.DD_GATHER_BULK if args.gather_mode == "bulk" else dd.DD_GATHER_LOADS
+    ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
+                     forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
+                     gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy)
+    budget = int(available_host_bytes() * 0.6 / max(1, world))
+    store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, host_budget_bytes=budget,
+                      log=log if rank == 0 else None)
+    store.bind(ctx)
+    if rank == 0:
+        log(f"{w.name}: host store {store.host_bytes / 2**30:.1f} GiB pinned in {store.n_phys} physical layer(s), "
+            f"built in {store.build_seconds:.1f} s; ring {ctx.ring_bytes() / 2**20:.0f} MiB, scratch {ctx.scratch_bytes() / 2**20:.1f} MiB")
+
+    # queries of every step (fresh each step), resident in HBM and also in pinned host memory for the e2e leg
+    n_q = W + K
+    q_host = torch.empty((n_q, L, B, 2, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, pin_memory=True)
+    for t in range(n_q):
+        for l in range(L):
+            q_host[t, l] = wl.queries(w, t, l)
+    q_dev = q_host.cuda()
+    q_init = torch.stack([wl.queries(w, -1, l)[:, 1] for l in range(L)]).cuda()
+    outs = torch.zeros((L, B, 2, w.n_q_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+    out_host = torch.empty(outs.shape, dtype=torch.bfloat16, pin_memory=True)
+
+    # host-link peak: pinned cudaMemcpyAsync host->device, best of 6 at 256 MiB
+    hsrc = torch.empty(256 << 20, dtype=torch.uint8, pin_memory=True)
+    hdst = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    link_peak = 0.0
+    for _ in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        hdst.copy_(hsrc, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        link_peak = max(link_peak, hsrc.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del hsrc, hdst
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def run_steps(t_from, t_to, step_base):
+        for t in range(t_from, t_to):
+            for l in range(L):
+                ctx.decode_layer_step(step_base + t - t_from, l, q_dev[t, l], outs[l])
+
+    # ---- device-resident run: W warm-up steps, then exactly K timed steps
+    ctx.prime(q_init)
+    run_steps(0, W, 0)
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tail = torch.cuda.Event()
+    ev0.record(compute)
+    x0.record(copy)
+    run_steps(W, W + K, W)
+    x1.record(copy)
+    tail.record(copy)
+    compute.wait_event(tail)          # the timed region ends when both streams are done
+    ev1.record(compute)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms_total = ev0.elapsed_time(ev1)
+    copy_ms = x0.elapsed_time(x1)
+    code, detail = ctx.device_error()
+    if code != 0:
+        raise RuntimeError(f"device error {code} (detail {detail}) during the timed run")
+    t_ms = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_total = float(t_ms.item())
+    ms_per_step = ms_total / K
+    value = world * B * K / (ms_total * 1e-3)
+    n_gathers = K * L
+    gather_bytes = w.gathered_bytes_per_layer
+    gather_ms_live = copy_ms / n_gathers
+
+    # ---- end-to-end run: every step copies its queries from pinned host memory, reads the outputs back
+    ctx.sync()
+    ctx.prime(q_init)
+    q_step = torch.empty_like(q_dev[0])
+    done = torch.cuda.Event()
+    with torch.cuda.stream(compute):
+        for t in range(W):
+            q_step.copy_(q_host[t], non_blocking=True)
+            for l in range(L):
+                ctx.decode_layer_step(t, l, q_step[l], outs[l])
+            out_host.copy_(outs, non_blocking=True)
+            done.record(compute)
+            done.synchronize()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(compute)
+        for t in range(W, W + K):
+            q_step.copy_(q_host[t], non_blocking=True)
+            for l in range(L):
+                ctx.decode_layer_step(t, l, q_step[l], outs[l])
+            out_host.copy_(outs, non_blocking=True)
+            done.record(compute)
+            done.synchronize()            # the caller needs the step's result before the next step
+        tail.record(copy)
+        compute.wait_event(tail)
+        e1.record(compute)
+    barrier()
+    t_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    e2e_value = world * B * K / (float(t_ms.item()) * 1e-3)
+    q_bytes = q_step.numel() * 2
+    o_bytes = outs.numel() * 2
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "batch": B, "ctx": w.ctx, "budget": w.budget, "layers": L,
+                   "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "gather_mode": args.gather_mode,
+                   "host_store_gib": store.host_bytes / 2**30, "phys_layers": store.n_phys,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2: each layer streams its own 32 MiB of landmarks and 64 MiB of "
+                         "freshly gathered pages; the host store is never cached",
+                   "generator": {k: v for k, v in w.params().items() if k in (
+                       "structure", "planted_frac", "zipf_a", "topic_gain", "planted_noise", "query_topic", "seed")}},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": q_bytes + L * gather_bytes,
+                "d2h_bytes_per_step": o_bytes,
+                "note": "queries copied from pinned host memory and outputs read back every step, host waits for "
+                        "each step; the KV gather from the host store is part of the path in both numbers"},
+        "gpu_launches": K * L * 4,
+        "clocks": clocks,
+    }
+
+    if rank == 0:
+        us_layer = ms_per_step / L * 1e3
+        link_time_us = gather_bytes / (link_peak * 1e9) * 1e6
+        hbm_bytes = (B * w.n_kv_heads * w.n_pages * 256 * 1.125) + 2 * gather_bytes
+        hbm_time_us = hbm_bytes / (hbm_peak * 1e9) * 1e6
+        line["roofline"] = {
+            "kernel": "dd_gather_loads_kernel" if args.gather_mode == "loads" else "dd_gather_bulk_kernel",
+            "bound": "host_link", "achieved": gather_bytes / (gather_ms_live * 1e-3) / 1e9, "peak": link_peak,
+            "unit": "GB/s", "frac": gather_bytes / (gather_ms_live * 1e-3) / 1e9 / link_peak, "traffic": None,
+            "peak_source": "pinned cudaMemcpyAsync host->device, 256 MiB, best of 6, measured in this run",
+            "how": "gathered bytes per launch / (copy-stream span of the timed region / launches)",
+        }
+        line["layer_step"] = {"us_per_layer": us_layer, "roofline_us": max(link_time_us, hbm_time_us),
+                              "frac_of_roofline": max(link_time_us, hbm_time_us) / us_layer,
+                              "link_us": link_time_us, "hbm_us": hbm_time_us, "hbm_peak_gbs": hbm_peak,
+                              "hbm_peak_source": peak_src}
+        if not args.no_stages:
+            line["stages"] = stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, args, K, W)
+            st = line["stages"]
+            t_c = st["compute_only_us_per_layer"]
+            t_g = st["gather_us"]
+            line["layer_step"].update({
+                "exposed_transfer_us_per_layer": us_layer - t_c,
+                "hidden_fraction_raw": 1.0 - (us_layer - t_c) / t_g,
+                "hidden_fraction_bound": min(1.0, t_c / t_g),
+                "overlap_efficiency": (t_c + t_g - us_layer) / min(t_c, t_g)})
+            line["roofline_kernels"] = st.pop("roofline_kernels")
+    ctx.sync()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        log("timing the CPU oracle on a sample of the workload ...")
+        line["cpu_baseline"] = oracle_sample(w)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, args, K, W):
+    """Each kernel alone, CUDA events on its stream, median over rotating layers (set-up for the split of a
+    layer into select / gather / attention and for the per-kernel rooflines)."""
+    L, B = w.n_layers, w.batch
+    cs, xs = ctx.compute_stream, ctx.copy_stream
+    ctx.sync()
+    reps = max(8, min(64, 2 * L))
+    idx = torch.stack([ctx.get_indices(0, l) for l in range(L)])
+    tmp_idx = torch.empty_like(idx[0])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(stream, fn, pre=None):
+        ts = []
+        for i in range(reps + 3):
+            if pre:
+                pre(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn(i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return statistics.median(ts), min(ts)
+
+    sel_us, sel_min = timed(cs, lambda i: ctx.select_topk(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
+                                                           store.n_pages_dev, tmp_idx, None, stream=cs))
+    gat_us, gat_min = timed(xs, lambda i: ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev,
+                                                                  i % args.ring_depth, stream=xs))
+
+    def fill(i):
+        ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev, 0, stream=cs)
+
+    def fill_and_flush(i):
+        fill(i)
+        with torch.cuda.stream(cs):
+            flush.fill_(i & 255)
+
+    att_warm, _ = timed(cs, lambda i: ctx.sparse_decode_attn(q_dev[0, i % L], 0, idx[i % L], store.ctx_len_dev,
+                                                             outs[i % L], None, stream=cs), pre=fill)
+    att_cold, att_cold_min = timed(cs, lambda i: ctx.sparse_decode_attn(q_dev[0, i % L], 0, idx[i % L],
+                                                                        store.ctx_len_dev, outs[i % L], None, stream=cs),
+                                   pre=fill_and_flush)
+    # compute-only step: attention + selection of every layer with the slot already filled
+    fill(0)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_rep = 4
+    for r in range(n_rep + 1):
+        if r == 1:
+            e0.record(cs)
+        for l in range(L):
+            ctx.sparse_decode_attn(q_dev[0, l], 0, idx[l], store.ctx_len_dev, outs[l], None, stream=cs)
+            ctx.select_topk(q_dev[0, l], 1, store.landmarks[l], store.n_pages_dev, tmp_idx, None, stream=cs)
+    e1.record(cs)
+    torch.cuda.synchronize()
+    compute_only = e0.elapsed_time(e1) * 1e3 / (n_rep * L)
+    lm_bytes = B * w.n_kv_heads * w.n_pages * 256
+    sel_bytes = lm_bytes * 1.125          # landmarks once + fp32 logits written and read (4 heads x 4 B per 256 B row, twice)
+    gb = w.gathered_bytes_per_layer
+    return {
+        "select_us": sel_us, "gather_us": gat_us, "attn_us_l2_warm": att_warm, "attn_us_l2_flushed": att_cold,
+        "compute_only_us_per_layer": compute_only, "reps": reps,
+        "roofline_kernels": {
+            "select(dd_score_kernel+dd_topk_kernel)": {"bound": "hbm", "achieved": sel_bytes / (sel_us * 1e-6) / 1e9,
+                                                       "peak": hbm_peak, "unit": "GB/s",
+                                                       "frac": sel_bytes / (sel_us * 1e-6) / 1e9 / hbm_peak},
+            "dd_attn_kernel(l2 flushed)": {"bound": "hbm", "achieved": gb / (att_cold * 1e-6) / 1e9, "peak": hbm_peak,
+                                           "unit": "GB/s", "frac": gb / (att_cold * 1e-6) / 1e9 / hbm_peak},
+            "gather(alone)": {"bound": "host_link", "achieved": gb / (gat_us * 1e-6) / 1e9, "peak": link_peak,
+                              "unit": "GB/s", "frac": gb / (gat_us * 1e-6) / 1e9 / link_peak},
+        },
+    }
+
+
+if __name__ == "__main__":
+    main()
