@@ -19,7 +19,8 @@
  *     dd_device_error synchronise.
  *   - the scratch memory of a context is shared by its calls: calls of the same kind must
  *     be stream-ordered with respect to each other (the pipelined path does this itself).
- *   - bf16 tensors are dense, row-major in the index order written, 16-byte aligned.
+ *   - tensors are dense, row-major in the index order written; bf16 tensors 16-byte aligned,
+ *     int32 and fp32 arrays 4-byte aligned.
  *   - geometry supported by the kernels: head_dim 128, page_tokens 16,
  *     n_q_tokens * (n_q_heads / n_kv_heads) <= 8. Anything else is DD_ERR_INVALID_ARG.
  *

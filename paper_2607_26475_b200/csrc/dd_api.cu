@@ -268,10 +268,11 @@ extern "C" int dd_slot_ptr(dd_ctx* ctx, int slot, void** dev_out) {
 // ---------------------------------------------------------------------------------------------
 // pointer checks
 // ---------------------------------------------------------------------------------------------
-// Device pointer of the context's device (16-byte aligned), or failure.
-static int dd_check_dev(dd_ctx* ctx, const void* p, const char* what) {
+// Device pointer of the context's device, aligned for its element type (16 bytes for bf16 tensors, which
+// are read with 16-byte loads; 4 bytes for int32 / fp32 arrays), or failure.
+static int dd_check_dev(dd_ctx* ctx, const void* p, const char* what, int align = 16) {
   if (!p) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is NULL", what);
-  if (((uintptr_t)p) & 15) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is not 16-byte aligned", what);
+  if (((uintptr_t)p) & (uintptr_t)(align - 1)) return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s is not %d-byte aligned", what, align);
   cudaPointerAttributes a;
   cudaError_t e = cudaPointerGetAttributes(&a, p);
   if (e != cudaSuccess) { cudaGetLastError(); return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s: %s", what, cudaGetErrorString(e)); }
@@ -315,7 +316,7 @@ extern "C" int dd_build_landmarks(dd_ctx* ctx, const void* kv_layer, const int* 
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_build_landmarks: ctx is NULL");
   const void* kv_dev = nullptr;
   DD_TRY(dd_check_store(ctx, kv_layer, "kv_layer", &kv_dev));
-  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
   DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
   return dd_launch_build_landmarks(ctx, kv_dev, ctx_len, landmarks, (cudaStream_t)stream);
 }
@@ -327,9 +328,9 @@ extern "C" int dd_select_topk(dd_ctx* ctx, const void* q, int q_token, const voi
     return dd_fail(ctx, DD_ERR_INVALID_ARG, "q_token %d outside [0, %d)", q_token, ctx->cfg.n_q_tokens);
   DD_TRY(dd_check_dev(ctx, q, "q"));
   DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
-  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
-  DD_TRY(dd_check_dev(ctx, out_idx, "out_idx"));
-  if (out_scores) DD_TRY(dd_check_dev(ctx, out_scores, "out_scores"));
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
+  DD_TRY(dd_check_dev(ctx, out_idx, "out_idx", 4));
+  if (out_scores) DD_TRY(dd_check_dev(ctx, out_scores, "out_scores", 4));
   return dd_launch_select(ctx, q, q_token, ctx->cfg.n_q_tokens, landmarks, n_pages, out_idx, out_scores,
                           (cudaStream_t)stream);
 }
@@ -341,8 +342,8 @@ extern "C" int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, co
     return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
   const void* kv_dev = nullptr;
   DD_TRY(dd_check_store(ctx, host_kv_layer, "host_kv_layer", &kv_dev));
-  DD_TRY(dd_check_dev(ctx, idx, "idx"));
-  if (n_pages) DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
+  DD_TRY(dd_check_dev(ctx, idx, "idx", 4));
+  if (n_pages) DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
   return dd_launch_gather(ctx, kv_dev, idx, n_pages, ctx->ring + (size_t)slot * ctx->slot_bytes, (cudaStream_t)stream);
 }
 
@@ -352,10 +353,10 @@ extern "C" int dd_sparse_decode_attn(dd_ctx* ctx, const void* q, int slot, const
   if (slot < 0 || slot >= ctx->cfg.ring_depth)
     return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
   DD_TRY(dd_check_dev(ctx, q, "q"));
-  DD_TRY(dd_check_dev(ctx, idx, "idx"));
-  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  DD_TRY(dd_check_dev(ctx, idx, "idx", 4));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
   DD_TRY(dd_check_dev(ctx, out, "out"));
-  if (out_lse) DD_TRY(dd_check_dev(ctx, out_lse, "out_lse"));
+  if (out_lse) DD_TRY(dd_check_dev(ctx, out_lse, "out_lse", 4));
   return dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, idx, ctx_len, out, out_lse,
                         (cudaStream_t)stream);
 }
@@ -376,8 +377,8 @@ extern "C" int dd_bind(dd_ctx* ctx, const void* const* landmarks_per_layer, cons
     ctx->landmarks[l] = landmarks_per_layer[l];
     ctx->host_kv[l] = dv;
   }
-  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages"));
-  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len"));
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
   ctx->n_pages = n_pages;
   ctx->ctx_len = ctx_len;
   ctx->bound = true;
