@@ -183,6 +183,34 @@ int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* 
 /* Device address of the index set [B][Hkv][k] that attention uses at (step parity, layer). No copy. */
 int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx);
 
+/* ---- attention without any allocation ----------------------------------------------------------- */
+
+/* (The paper has no counterpart of this call; it exists for integration.)
+ * The same attention as dd_sparse_decode_attn, for callers that cannot allocate device memory and
+ * therefore cannot own a dd_ctx (dd_create allocates): code that runs inside another framework's
+ * memory plan, a process whose GPU memory is already fully handed to an arena, or a serving loop in
+ * which an allocation's implicit device synchronisation is not acceptable. The split-merge scratch
+ * lives in a fixed array of dd_static_scratch_capacity() bytes (8 MiB) inside the library image;
+ * every GPU that loads the library holds that array until the process exits.
+ *   - Nothing is allocated or freed: no cudaMalloc/cudaFree, no allocating library routine.
+ *   - The caller passes the gathered slot itself (dev bf16 [B][Hkv][2][k*T][d]) instead of a ring
+ *     slot number, and every other tensor as in dd_sparse_decode_attn.
+ *   - n_splits is explicit (1 <= n_splits <= k_pages). B * Hkv * n_splits * 4160 bytes (plus 4 bytes
+ *     per (request, KV head)) must fit the array; larger requests fail with DD_ERR_INVALID_ARG and a
+ *     message that states both sizes. n_splits = 1 needs almost nothing.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+ *     device current) and remembers it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *     clears the arrival counters it needs on `stream` before the kernel. Two calls that overlap on the
+ *     GPU (different streams, no ordering between them) race on the array and give wrong results:
+ *     order them.
+ * Asynchronous on `stream`. Returns DD_OK or DD_ERR_INVALID_ARG / DD_ERR_CUDA; the message is
+ * available from dd_last_error_message(NULL) on the calling thread. */
+size_t dd_static_scratch_capacity(void);
+int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_heads, int head_dim, int page_tokens,
+                                 int k_pages, int n_q_tokens, int n_splits, const void* q, const void* slot,
+                                 const int* idx, const int* ctx_len, void* out, float* out_lse, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ EXPORTS = [
     "dd_create", "dd_destroy", "dd_slot_bytes", "dd_ring_bytes", "dd_scratch_bytes", "dd_slot_ptr",
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
-    "dd_decode_layer_step", "dd_get_indices",
+    "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
 ]
 
 
@@ -78,6 +78,9 @@ def _load() -> C.CDLL:
     lib.dd_prime.argtypes = [vp, vp]
     lib.dd_decode_layer_step.argtypes = [vp, ip, ip, vp, vp]
     lib.dd_get_indices.argtypes = [vp, ip, ip, C.POINTER(vp)]
+    lib.dd_static_scratch_capacity.argtypes = []
+    lib.dd_static_scratch_capacity.restype = C.c_size_t
+    lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7
     return lib
 
 
@@ -113,6 +116,19 @@ def _stream(s) -> int:
     if isinstance(s, int):
         return s
     return s.cuda_stream
+
+
+def sparse_decode_attn_static(q, slot, idx, ctx_len, out, out_lse=None, *, n_splits=1, page_tokens=16, stream=None):
+    """Attention over a gathered slot without a context and without any allocation: for callers that are
+    not allowed to allocate device memory. The library's built-in scratch array (8 MiB per GPU) is shared
+    by every call on the device, so calls must not overlap on the GPU; the first call on a device should
+    come before any stream capture. q [B, Tq, Hq, d], slot [B, Hkv, 2, k*T, d], idx [B, Hkv, k]."""
+    B, Tq, Hq, d = q.shape
+    Hkv, k = idx.shape[1], idx.shape[2]
+    rc = lib.dd_sparse_decode_attn_static(B, Hq, Hkv, d, page_tokens, k, Tq, n_splits, _ptr(q), _ptr(slot), _ptr(idx),
+                                          _ptr(ctx_len), _ptr(out), _ptr(out_lse), _stream(stream))
+    if rc != DD_OK:
+        raise DDError(rc, lib.dd_last_error_message(None).decode())
 
 
 class Context:

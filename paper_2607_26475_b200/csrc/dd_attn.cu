@@ -256,3 +256,93 @@ int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx,
   DD_CUDA_TRY(ctx, cudaGetLastError());
   return DD_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the attention entry point.
+//
+// Some callers must not allocate device memory: code running between other libraries' memory pools,
+// a plug-in that was handed every byte it may touch, a process that has already given the whole GPU
+// to an arena allocator, or a latency-critical loop where an allocation (which can synchronise the
+// device) is not acceptable. A dd_ctx cannot serve them, because dd_create allocates the split-merge
+// scratch. This entry point keeps that scratch in a fixed array inside the library image instead.
+//
+// The array's name below is only a host-side handle in host code: passing it to a kernel would hand
+// the kernel a host address. Its device address is looked up once per device with
+// cudaGetSymbolAddress (by the first call on that device) and that address is what the kernel gets.
+// ------------------------------------------------------------------------------------------------
+#include <mutex>
+
+constexpr size_t DD_STATIC_SCRATCH_BYTES = (size_t)8 << 20;   // held by every GPU that loads the library
+static __device__ __align__(256) unsigned char dd_static_scratch[DD_STATIC_SCRATCH_BYTES];
+
+constexpr int DD_STATIC_MAX_DEVICES = 64;
+static unsigned char* g_static_scratch_addr[DD_STATIC_MAX_DEVICES];   // device address per device, 0 = not set up
+static std::mutex g_static_scratch_mutex;
+
+static size_t dd_static_need(int batch, int n_kv_heads, int n_splits, size_t* off_ml, size_t* off_ticket) {
+  const size_t bg = (size_t)batch * n_kv_heads;
+  const size_t part_o = (bg * n_splits * ATTN_ROWS * DD_D * sizeof(float) + 255) & ~(size_t)255;
+  const size_t part_ml = (bg * n_splits * ATTN_ROWS * sizeof(float2) + 255) & ~(size_t)255;
+  const size_t ticket = (bg * sizeof(unsigned int) + 255) & ~(size_t)255;
+  if (off_ml) *off_ml = part_o;
+  if (off_ticket) *off_ticket = part_o + part_ml;
+  return part_o + part_ml + ticket;
+}
+
+extern "C" size_t dd_static_scratch_capacity(void) { return DD_STATIC_SCRATCH_BYTES; }
+
+extern "C" int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_heads, int head_dim, int page_tokens,
+                                            int k_pages, int n_q_tokens, int n_splits, const void* q,
+                                            const void* slot, const int* idx, const int* ctx_len, void* out,
+                                            float* out_lse, void* stream) {
+  if (head_dim != DD_D || page_tokens != DD_T)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: head_dim must be 128 and page_tokens 16");
+  if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || k_pages < 1 || n_q_tokens < 1 ||
+      n_q_tokens > 2 || n_q_tokens * (n_q_heads / n_kv_heads) > ATTN_ROWS)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: unsupported geometry");
+  if (n_splits < 1 || n_splits > k_pages)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: need 1 <= n_splits <= k_pages");
+  if (!q || !slot || !idx || !ctx_len || !out)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: NULL tensor");
+  if ((((uintptr_t)q) | ((uintptr_t)slot) | ((uintptr_t)out)) & 15)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: bf16 tensors must be 16-byte aligned");
+  size_t off_ml = 0, off_ticket = 0;
+  const size_t need = dd_static_need(batch, n_kv_heads, n_splits, &off_ml, &off_ticket);
+  if (need > DD_STATIC_SCRATCH_BYTES)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG,
+                   "dd_sparse_decode_attn_static: batch %d x kv heads %d x splits %d needs %zu bytes of scratch, the "
+                   "built-in array holds %zu; use fewer splits or a dd_ctx",
+                   batch, n_kv_heads, n_splits, need, (size_t)DD_STATIC_SCRATCH_BYTES);
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= DD_STATIC_MAX_DEVICES)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: device ordinal %d not supported", dev);
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+      // once per device, with that device current: the device address of this device's copy of the array
+      void* p = nullptr;
+      e = cudaGetSymbolAddress(&p, dd_static_scratch);
+      if (e != cudaSuccess || !p)
+        return dd_fail(nullptr, DD_ERR_CUDA, "cudaGetSymbolAddress(dd_static_scratch): %s", cudaGetErrorString(e));
+      g_static_scratch_addr[dev] = (unsigned char*)p;
+    }
+    base = g_static_scratch_addr[dev];
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned int* ticket = (unsigned int*)(base + off_ticket);
+  // the array keeps whatever the previous call (or an interrupted one) left: the arrival counters must start at zero
+  e = cudaMemsetAsync(ticket, 0, (size_t)batch * n_kv_heads * sizeof(unsigned int), st);
+  if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  const int pps = (k_pages + n_splits - 1) / n_splits;
+  dim3 grid(n_splits, n_kv_heads, batch);
+  dd_attn_kernel<<<grid, ATTN_THREADS, 0, st>>>((const __nv_bfloat16*)q, (const char*)slot, idx, ctx_len,
+                                                (__nv_bfloat16*)out, out_lse, (float*)base, (float2*)(base + off_ml),
+                                                ticket, n_kv_heads, n_q_heads / n_kv_heads, n_q_tokens, k_pages,
+                                                n_splits, pps);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "dd_attn_kernel launch: %s", cudaGetErrorString(e));
+  return DD_OK;
+}

@@ -1,0 +1,69 @@
+"""The allocation-free attention entry point against the context-based one.
+
+Callers that may not allocate device memory (they run inside someone else's memory plan, or must not
+trigger the device synchronisation an allocation can cause) use dd_sparse_decode_attn_static, whose
+scratch is a fixed array inside the library. It must give the same result as dd_sparse_decode_attn on
+the same gathered slot, call after call, although every call reuses (and finds the leftovers of the
+previous call in) the same array. Collected last on purpose: a run that stops at the first failure has
+then already run every other test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from tests._util import ATTN_MAX_ABS, ATTN_MEAN_ABS, f32
+
+pytestmark = pytest.mark.gpu
+
+HKV, D, T = 8, 128, 16
+
+
+def _case(dd, seed, B, P, k, splits_ctx, splits_static, ctx_len):
+    g = torch.Generator().manual_seed(seed)
+    kv = torch.randn(B, HKV, P, 2, T, D, generator=g).to(torch.bfloat16).pin_memory()
+    q = torch.randn(B, 2, 32, D, generator=g).to(torch.bfloat16).cuda()
+    idx = torch.stack([torch.stack([torch.randperm(P, generator=g)[:k].sort().values for _ in range(HKV)])
+                       for _ in range(B)]).to(torch.int32).cuda()
+    cl = torch.tensor(ctx_len, dtype=torch.int32).cuda()
+    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, attn_splits=splits_ctx)
+    c.gather_kv_from_host(kv, idx, None, 0)
+    want = torch.empty((B, 2, 32, D), dtype=torch.bfloat16, device="cuda")
+    want_lse = torch.empty((B, 2, 32), dtype=torch.float32, device="cuda")
+    c.sparse_decode_attn(q, 0, idx, cl, want, want_lse)
+    slot = c.slot_tensor(0)                               # the caller of the static entry point owns the slot
+    got = torch.full_like(want, 3.0)
+    got_lse = torch.zeros_like(want_lse)
+    dd.sparse_decode_attn_static(q, slot, idx, cl, got, got_lse, n_splits=splits_static)
+    torch.cuda.synchronize()
+    assert c.device_error() == (0, 0)
+    c.close()
+    err = np.abs(f32(got).astype(np.float64) - f32(want).astype(np.float64))
+    assert err.max() <= ATTN_MAX_ABS and err.mean() <= ATTN_MEAN_ABS, (err.max(), err.mean())
+    np.testing.assert_allclose(got_lse.cpu().numpy(), want_lse.cpu().numpy(), atol=2e-3, rtol=1e-4)
+    return err.max()
+
+
+def test_static_entry_point_matches_the_context_entry_point_on_consecutive_calls():
+    from paper_2607_26475_b200 import binding as dd
+    assert dd.lib.dd_static_scratch_capacity() == 8 << 20
+    # two calls in a row with different shapes and split counts: the second finds the first one's leftovers
+    e1 = _case(dd, 1, B=3, P=200, k=64, splits_ctx=4, splits_static=4, ctx_len=[3200, 3190, 1700])
+    e2 = _case(dd, 2, B=2, P=150, k=37, splits_ctx=1, splits_static=5, ctx_len=[2400, 2399])
+    e3 = _case(dd, 3, B=3, P=200, k=64, splits_ctx=4, splits_static=4, ctx_len=[3200, 3190, 1700])
+    assert e1 == 0.0 and e3 == 0.0          # same split geometry gives the same bits as the context path
+    assert e2 <= ATTN_MAX_ABS
+
+
+def test_static_entry_point_rejects_what_does_not_fit():
+    from paper_2607_26475_b200 import binding as dd
+    B, k = 64, 128
+    q = torch.zeros((B, 2, 32, D), dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros((B, HKV, k), dtype=torch.int32, device="cuda")
+    cl = torch.full((B,), k * T, dtype=torch.int32, device="cuda")
+    slot = torch.zeros((1,), dtype=torch.bfloat16, device="cuda")       # never touched: the call must fail first
+    with pytest.raises(dd.DDError) as e:
+        dd.sparse_decode_attn_static(q, slot, idx, cl, q.clone(), n_splits=8)   # 64 * 8 * 8 * 4160 B > 8 MiB
+    assert e.value.code == dd.DD_ERR_INVALID_ARG and "8388608" in str(e.value)
+    with pytest.raises(dd.DDError) as e:
+        dd.sparse_decode_attn_static(q, slot, idx, cl, q.clone(), n_splits=k + 1)
+    assert e.value.code == dd.DD_ERR_INVALID_ARG
