@@ -36,7 +36,7 @@ def log(msg):
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=2, help="workload number (2 = batch 8, 32K context, budget 2048)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -105,7 +105,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(w, n_layers_cap=4, min_seconds=8.0):
+def oracle_sample(w, n_layers_cap=32, min_seconds=10.0):
     """Times the oracle, as it stands, on whole layers of the workload (all requests, one step):
     selection from the speculated token, page gather, attention of both tokens. Returns tok/s scaled to
     a full step of w.n_layers layers."""
@@ -251,10 +251,15 @@ def main():
                 ctx.decode_layer_step(step_base + t - t_from, l, q_dev[t, l], outs[l])
 
     # ---- device-resident run: W warm-up steps, then exactly K timed steps
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     ctx.prime(q_init)
     run_steps(0, W, 0)
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        t_wait = time.time()
+        while not sampler.rows and time.time() - t_wait < 3.0:     # nvidia-smi takes a moment to start
+            time.sleep(0.05)
+        sampler.rows.clear()                                       # keep only samples of the timed region
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     tail = torch.cuda.Event()
@@ -376,8 +381,10 @@ def main():
 
 
 def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, args, K, W):
-    """Each kernel alone, CUDA events on its stream, median over rotating layers (set-up for the split of a
-    layer into select / gather / attention and for the per-kernel rooflines)."""
+    """Each kernel alone, CUDA events on its stream around batches of launches (the split of a layer into
+    select / gather / attention and the per-kernel rooflines). Selection and gather rotate over the layers
+    (every launch reads landmarks / host pages no earlier launch left in L2); attention is timed both on an
+    L2-warm slot and with L2 flushed before every launch."""
     L, B = w.n_layers, w.batch
     cs, xs = ctx.compute_stream, ctx.copy_stream
     ctx.sync()
@@ -387,39 +394,43 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
     def timed(stream, fn, pre=None):
-        ts = []
-        for i in range(reps + 3):
-            if pre:
-                pre(i)
+        """Average device time of fn over `reps` launches enqueued back to back on `stream` (no host
+        synchronisation in between, as in the pipeline); `pre` runs before every launch and its own cost,
+        measured the same way, is subtracted."""
+        def batch(with_fn):
+            for i in range(3):
+                if pre:
+                    pre(i)
+                if with_fn:
+                    fn(i)
+            torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            fn(i)
+            for i in range(reps):
+                if pre:
+                    pre(i)
+                if with_fn:
+                    fn(i)
             e1.record(stream)
             torch.cuda.synchronize()
-            if i >= 3:
-                ts.append(e0.elapsed_time(e1) * 1e3)
-        return statistics.median(ts), min(ts)
+            return e0.elapsed_time(e1) * 1e3 / reps
+        total = batch(True)
+        return total - (batch(False) if pre else 0.0)
 
-    sel_us, sel_min = timed(cs, lambda i: ctx.select_topk(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
-                                                           store.n_pages_dev, tmp_idx, None, stream=cs))
-    gat_us, gat_min = timed(xs, lambda i: ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev,
-                                                                  i % args.ring_depth, stream=xs))
+    sel_us = timed(cs, lambda i: ctx.select_topk(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
+                                                 store.n_pages_dev, tmp_idx, None, stream=cs))
+    gat_us = timed(xs, lambda i: ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev,
+                                                         i % args.ring_depth, stream=xs))
+    ctx.gather_kv_from_host(store.kv[0], idx[0], store.n_pages_dev, 0, stream=cs)
 
-    def fill(i):
-        ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev, 0, stream=cs)
-
-    def fill_and_flush(i):
-        fill(i)
+    def flush_l2(i):
         with torch.cuda.stream(cs):
             flush.fill_(i & 255)
 
-    att_warm, _ = timed(cs, lambda i: ctx.sparse_decode_attn(q_dev[0, i % L], 0, idx[i % L], store.ctx_len_dev,
-                                                             outs[i % L], None, stream=cs), pre=fill)
-    att_cold, att_cold_min = timed(cs, lambda i: ctx.sparse_decode_attn(q_dev[0, i % L], 0, idx[i % L],
-                                                                        store.ctx_len_dev, outs[i % L], None, stream=cs),
-                                   pre=fill_and_flush)
+    attn = lambda i: ctx.sparse_decode_attn(q_dev[0, 0], 0, idx[0], store.ctx_len_dev, outs[0], None, stream=cs)
+    att_warm = timed(cs, attn)
+    att_cold = timed(cs, attn, pre=flush_l2)
     # compute-only step: attention + selection of every layer with the slot already filled
-    fill(0)
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n_rep = 4
@@ -427,7 +438,7 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
         if r == 1:
             e0.record(cs)
         for l in range(L):
-            ctx.sparse_decode_attn(q_dev[0, l], 0, idx[l], store.ctx_len_dev, outs[l], None, stream=cs)
+            ctx.sparse_decode_attn(q_dev[0, l], 0, idx[0], store.ctx_len_dev, outs[l], None, stream=cs)
             ctx.select_topk(q_dev[0, l], 1, store.landmarks[l], store.n_pages_dev, tmp_idx, None, stream=cs)
     e1.record(cs)
     torch.cuda.synchronize()

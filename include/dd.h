@@ -65,7 +65,7 @@ typedef struct dd_config {
   int ring_depth;            /* D >= 2 (2 = the two-buffer scheme) */
   int gather_mode;           /* DD_GATHER_LOADS or DD_GATHER_BULK */
   int gather_ctas;           /* thread blocks the gather may occupy; 0 = library default */
-  int attn_splits;           /* splits of the gathered set per (request, KV head); 0 = chosen from the SM count */
+  int attn_splits;           /* blocks per (request, KV head) in attention, <= 64 or a multiple of 8 up to 512; 0 = automatic */
   void* compute_stream;      /* cudaStream_t used by the pipelined calls for attention and selection */
   void* copy_stream;         /* cudaStream_t used by the pipelined calls for the gather */
   void* ring_mem;            /* optional caller-owned ring of dd_ring_bytes(); NULL = library allocates */
@@ -195,7 +195,7 @@ int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx)
  *   - Nothing is allocated or freed: no cudaMalloc/cudaFree, no allocating library routine.
  *   - The caller passes the gathered slot itself (dev bf16 [B][Hkv][2][k*T][d]) instead of a ring
  *     slot number, and every other tensor as in dd_sparse_decode_attn.
- *   - n_splits is explicit (1 <= n_splits <= k_pages). B * Hkv * n_splits * 4160 bytes (plus 4 bytes
+ *   - n_splits is explicit (1 <= n_splits <= min(k_pages, 64)). B * Hkv * n_splits * 4160 bytes (plus 4 bytes
  *     per (request, KV head)) must fit the array; larger requests fail with DD_ERR_INVALID_ARG and a
  *     message that states both sizes. n_splits = 1 needs almost nothing.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that

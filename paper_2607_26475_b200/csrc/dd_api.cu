@@ -57,23 +57,38 @@ static const char* dd_check_config(const dd_config* c) {
   if (c->ring_depth < 2 || c->ring_depth > DD_MAX_RING) return "ring_depth must be in [2, 8]";
   if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK) return "unknown gather_mode";
   if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
+  if (c->attn_splits > 512) return "attn_splits must be <= 512";
+  if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";
   if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
   if ((long long)c->batch * c->n_kv_heads * c->max_pages > 0x7fffffffLL) return "too many pages";
   return nullptr;
 }
 
-static int dd_resolve_splits(const dd_config* c, int sm_count) {
-  int S = c->attn_splits;
+// Blocks per (request, KV head) and how many of them form a thread-block cluster. Automatic choice: one
+// wave of blocks (the attention kernel keeps four per SM resident), at least four pages (one per warp) in a
+// split, clusters of up to eight blocks so that up to eight splits merge without touching global memory.
+static int dd_resolve_splits(const dd_config* c, int sm_count, int* cluster_out) {
+  int S = c->attn_splits, C = 1;
   if (S <= 0) {
-    // enough blocks for about four per SM, but at least four pages (one per warp) in a split
     const int problems = c->batch * c->n_kv_heads;
-    S = (4 * sm_count + problems - 1) / problems;
-    const int s_max = c->k_pages / 4 > 0 ? c->k_pages / 4 : 1;
-    if (S > s_max) S = s_max;
-    if (S > 64) S = 64;
+    int target = (4 * sm_count) / problems;
+    const int t_max = c->k_pages / 4 > 0 ? c->k_pages / 4 : 1;
+    if (target > t_max) target = t_max;
+    if (target < 1) target = 1;
+    if (target >= 8) {
+      int groups = target / 8;
+      if (groups > 64) groups = 64;
+      C = 8;
+      S = 8 * groups;
+    } else {
+      C = target >= 4 ? 4 : (target >= 2 ? 2 : 1);
+      S = C;
+    }
+  } else {
+    if (S > c->k_pages) S = c->k_pages;
+    C = (S % 8 == 0) ? 8 : (S % 4 == 0) ? 4 : (S % 2 == 0) ? 2 : 1;
   }
-  if (S > c->k_pages) S = c->k_pages;
-  if (S < 1) S = 1;
+  if (cluster_out) *cluster_out = C;
   return S;
 }
 
@@ -113,7 +128,7 @@ extern "C" size_t dd_slot_bytes(const dd_config* c) {
 extern "C" size_t dd_ring_bytes(const dd_config* c) { return dd_slot_bytes(c) * (c ? (size_t)c->ring_depth : 0); }
 extern "C" size_t dd_scratch_bytes(const dd_config* c) {
   if (dd_check_config(c)) return 0;
-  return dd_compute_sizes(c, dd_resolve_splits(c, dd_sm_count())).total();
+  return dd_compute_sizes(c, dd_resolve_splits(c, dd_sm_count(), nullptr)).total();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -154,7 +169,7 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
   ctx->n_rows = cfg->n_q_tokens * ctx->G;
   ctx->score_tiles = (cfg->max_pages + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
-  ctx->attn_splits = dd_resolve_splits(cfg, ctx->sm_count);
+  ctx->attn_splits = dd_resolve_splits(cfg, ctx->sm_count, &ctx->attn_cluster);
   ctx->slot_bytes = dd_slot_bytes(cfg);
   const dd_sizes z = dd_compute_sizes(cfg, ctx->attn_splits);
 

@@ -14,11 +14,35 @@
 //   * for O^T the rows of the MMA (channels) may be assigned freely, so a thread takes 8 consecutive
 //     channels of tokens 2t, 2t+1, 2t+8, 2t+9 and pairs neighbouring tokens with byte permutes;
 //   * P^T goes from accumulator layout to B-operand layout with one 8x8 matrix transpose per half page.
+#include <cooperative_groups.h>
+
 #include "dd_common.cuh"
+
+// Optional per-block timeline for tuning (compile with -DDD_TRACE; never in the shipped library):
+// mark i of block (x, y, z) is the global nanosecond timer when thread 0 passed it.
+#ifdef DD_TRACE
+__device__ unsigned long long dd_trace_buf[1 << 16][8];
+#define DD_TRACE_MARK(i)                                                                                     \
+  do {                                                                                                       \
+    if (threadIdx.x == 0) {                                                                                  \
+      unsigned long long t__;                                                                                \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));                                                \
+      dd_trace_buf[(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x][i] = t__;                 \
+    }                                                                                                        \
+  } while (0)
+extern "C" int dd_trace_read(unsigned long long* host, size_t bytes) {
+  return (int)cudaMemcpyFromSymbol(host, dd_trace_buf, bytes);
+}
+#else
+#define DD_TRACE_MARK(i)
+#endif
 
 constexpr int ATTN_WARPS = 4;
 constexpr int ATTN_THREADS = ATTN_WARPS * 32;
 constexpr int ATTN_ROWS = 8;       // query rows per KV head the MMA shape carries
+constexpr int ATTN_MAX_SPLITS = 64;
+constexpr int ATTN_MAX_CLUSTER = 8;
+constexpr int ATTN_OPAD = 9;       // row pitch (floats) of the per-warp O^T staging: conflict-free reads, 2-way writes
 
 __device__ __forceinline__ uint32_t dd_movmatrix_trans(uint32_t a) {
   uint32_t d;
@@ -31,11 +55,38 @@ __device__ __forceinline__ uint32_t dd_pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
+// K rows gl and gl+8 of a page: channels [32kk + 8t, +8) for kk = 0..3
+__device__ __forceinline__ void dd_load_k(const char* kp, int gl, int t, uint4 (&klo)[4], uint4 (&khi)[4]) {
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    klo[kk] = dd_ld_stream(kp + gl * DD_ROW_BYTES + (kk * 4 + t) * 16);
+    khi[kk] = dd_ld_stream(kp + (gl + 8) * DD_ROW_BYTES + (kk * 4 + t) * 16);
+  }
+}
+
+// V tokens 2t, 2t+1, 2t+8, 2t+9 of a page: channels [8gl, 8gl+8) and [64+8gl, 64+8gl+8)
+__device__ __forceinline__ void dd_load_v(const char* vp, int gl, int t, uint4 (&v)[4][2]) {
+#pragma unroll
+  for (int tk = 0; tk < 4; ++tk) {
+    const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) v[tk][c] = dd_ld_stream(vp + tok * DD_ROW_BYTES + (c * 64 + gl * 8) * 2);
+  }
+}
+
+__device__ __forceinline__ uint32_t dd_word(const uint4& v, int w) {
+  return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+}
+
+// Grid (n_splits, KV head, request), launched with thread-block clusters of `cluster` blocks along x
+// (n_splits = cluster * n_groups). The blocks of a cluster merge through distributed shared memory;
+// when a (request, KV head) has several clusters, each publishes a partial to global scratch and the
+// last one to arrive merges them (arrival counter, no waiting).
+__global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     const __nv_bfloat16* __restrict__ q, const char* __restrict__ slot, const int* __restrict__ idx,
     const int* __restrict__ ctx_len, __nv_bfloat16* __restrict__ out, float* __restrict__ out_lse,
     float* __restrict__ part_o, float2* __restrict__ part_ml, unsigned int* __restrict__ ticket, int Hkv, int G, int Tq,
-    int k, int n_splits, int pages_per_split) {
+    int k, int n_splits, int pages_per_split, int cluster) {
   const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gl = lane >> 2, t = lane & 3;
@@ -43,11 +94,14 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
   const int n_rows = Tq * G;
   const size_t bg = (size_t)b * Hkv + g;
 
-  __shared__ float sm_o[ATTN_WARPS][ATTN_ROWS][DD_D];
+  __shared__ float sm_o[ATTN_WARPS][DD_D][ATTN_OPAD];   // per-warp O^T, [channel][row]
   __shared__ float2 sm_ml[ATTN_WARPS][ATTN_ROWS];
   __shared__ float sm_scale[ATTN_WARPS][ATTN_ROWS];
+  __shared__ float blk_o[ATTN_ROWS][DD_D];              // block result, read by the cluster's other blocks
+  __shared__ float2 blk_ml[ATTN_ROWS];
   __shared__ int sm_last;
 
+  DD_TRACE_MARK(0);
   // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G)
   uint4 qf[4];
   if (gl < n_rows) {
@@ -75,28 +129,17 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
 
   const int p_begin = split * pages_per_split;
   const int p_end = min(k, p_begin + pages_per_split);
-  for (int j = p_begin + warp; j < p_end; j += ATTN_WARPS) {
-    // ---- loads: K rows gl and gl+8; V tokens 2t, 2t+1, 2t+8, 2t+9, channels [8gl, 8gl+8) and [64+8gl, ..)
-    const char* kp = kbase + (size_t)j * DD_HALF_PAGE_BYTES;
-    const char* vp = vbase + (size_t)j * DD_HALF_PAGE_BYTES;
-    uint4 klo[4], khi[4];
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      klo[kk] = dd_ld_stream(kp + gl * DD_ROW_BYTES + (kk * 4 + t) * 16);
-      khi[kk] = dd_ld_stream(kp + (gl + 8) * DD_ROW_BYTES + (kk * 4 + t) * 16);
-    }
-    uint32_t v[4][2][4];
-#pragma unroll
-    for (int tk = 0; tk < 4; ++tk) {
-      const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        const uint4 w = dd_ld_stream(vp + tok * DD_ROW_BYTES + (c * 64 + gl * 8) * 2);
-        v[tk][c][0] = w.x; v[tk][c][1] = w.y; v[tk][c][2] = w.z; v[tk][c][3] = w.w;
-      }
-    }
-    const int page = idx_bg[j];
-
+  int j = p_begin + warp;
+  uint4 klo[4], khi[4], v[4][2];
+  int page = 0;
+  if (j < p_end) {
+    dd_load_k(kbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
+    dd_load_v(vbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, v);
+    page = idx_bg[j];
+  }
+  while (j < p_end) {
+    const int jn = j + ATTN_WARPS;
+    const bool has_next = jn < p_end;
     // ---- S^T = K q^T
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -104,6 +147,9 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
       dd_mma_bf16(acc, klo[kk].x, khi[kk].x, klo[kk].y, khi[kk].y, qf[kk].x, qf[kk].y);
       dd_mma_bf16(acc, klo[kk].z, khi[kk].z, klo[kk].w, khi[kk].w, qf[kk].z, qf[kk].w);
     }
+    // the K fragments are consumed: the next page's K goes into the same registers while this page finishes
+    if (has_next) dd_load_k(kbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
+    const int page_next = has_next ? idx_bg[jn] : 0;
     // acc[0], acc[1]: token gl, columns 2t, 2t+1; acc[2], acc[3]: token gl+8
 #pragma unroll
     for (int i = 0; i < 4; ++i) acc[i] *= scale_log2;
@@ -142,13 +188,18 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
     for (int i = 0; i < 8; ++i) {
       const int w = i >> 1;
       const uint32_t sel = (i & 1) ? 0x7632u : 0x5410u;
-      const uint32_t a0 = __byte_perm(v[0][0][w], v[1][0][w], sel);
-      const uint32_t a1 = __byte_perm(v[0][1][w], v[1][1][w], sel);
-      const uint32_t a2 = __byte_perm(v[2][0][w], v[3][0][w], sel);
-      const uint32_t a3 = __byte_perm(v[2][1][w], v[3][1][w], sel);
+      const uint32_t a0 = __byte_perm(dd_word(v[0][0], w), dd_word(v[1][0], w), sel);
+      const uint32_t a1 = __byte_perm(dd_word(v[0][1], w), dd_word(v[1][1], w), sel);
+      const uint32_t a2 = __byte_perm(dd_word(v[2][0], w), dd_word(v[3][0], w), sel);
+      const uint32_t a3 = __byte_perm(dd_word(v[2][1], w), dd_word(v[3][1], w), sel);
       dd_mma_bf16(o[i], a0, a1, a2, a3, pb0, pb1);
     }
+    if (has_next) dd_load_v(vbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, v);
+    if (j == p_begin + warp) DD_TRACE_MARK(1);
+    page = page_next;
+    j = jn;
   }
+  DD_TRACE_MARK(2);
   // l over the 8 row groups of the warp
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -163,10 +214,10 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    sm_o[warp][2 * t][8 * gl + i] = o[i][0];
-    sm_o[warp][2 * t + 1][8 * gl + i] = o[i][1];
-    sm_o[warp][2 * t][64 + 8 * gl + i] = o[i][2];
-    sm_o[warp][2 * t + 1][64 + 8 * gl + i] = o[i][3];
+    sm_o[warp][8 * gl + i][2 * t] = o[i][0];
+    sm_o[warp][8 * gl + i][2 * t + 1] = o[i][1];
+    sm_o[warp][64 + 8 * gl + i][2 * t] = o[i][2];
+    sm_o[warp][64 + 8 * gl + i][2 * t + 1] = o[i][3];
   }
   __syncthreads();
   if (threadIdx.x < ATTN_ROWS) {
@@ -181,16 +232,17 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
       sm_scale[w][n] = sc;
       L += sm_ml[w][n].y * sc;
     }
-    sm_ml[0][n] = make_float2(M, L);             // block result, read after the next barrier
+    blk_ml[n] = make_float2(M, L);
   }
   __syncthreads();
+  DD_TRACE_MARK(3);
   const int d = threadIdx.x;                     // one channel per thread, all rows
   float ob[ATTN_ROWS];
 #pragma unroll
   for (int n = 0; n < ATTN_ROWS; ++n) {
     float a = 0.f;
 #pragma unroll
-    for (int w = 0; w < ATTN_WARPS; ++w) a += sm_o[w][n][d] * sm_scale[w][n];
+    for (int w = 0; w < ATTN_WARPS; ++w) a += sm_o[w][d][n] * sm_scale[w][n];
     ob[n] = a;
   }
 
@@ -199,7 +251,7 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
     for (int n = 0; n < ATTN_ROWS; ++n) {
       if (n < n_rows) {
         const int tq = n / G, hh = n - tq * G;
-        const float2 ml = sm_ml[0][n];
+        const float2 ml = blk_ml[n];
         const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
         out[row * DD_D + d] = __float2bfloat16_rn(ml.y > 0.f ? ob[n] / ml.y : 0.f);
         if (out_lse && d == 0) out_lse[row] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
@@ -208,52 +260,153 @@ __global__ void __launch_bounds__(ATTN_THREADS) dd_attn_kernel(
     return;
   }
 
-  // ---- several splits: publish the partial, the last block to arrive merges
-  {
-    float* po = part_o + ((bg * n_splits + split) * ATTN_ROWS) * DD_D;
+  const int n_groups = n_splits / cluster;       // clusters per (request, KV head)
+  const int group = split / cluster;
+  if (cluster > 1) {
+    // ---- merge the blocks of the cluster through distributed shared memory: block `rank` reduces the
+    // channels [rank*128/cluster, (rank+1)*128/cluster) of all rows over every block of the cluster
+    namespace cg = cooperative_groups;
+    cg::cluster_group cl = cg::this_cluster();
+    const int rank = (int)cl.block_rank();
+#pragma unroll
+    for (int n = 0; n < ATTN_ROWS; ++n) blk_o[n][d] = ob[n];
+    cl.sync();
+    const int ch = DD_D / cluster;               // channels per block
+    for (int e = threadIdx.x; e < ATTN_ROWS * ch; e += ATTN_THREADS) {
+      const int n = e / ch, dd = rank * ch + (e - n * ch);
+      float ms[ATTN_MAX_CLUSTER], ls[ATTN_MAX_CLUSTER], os[ATTN_MAX_CLUSTER];
+      float M = -INFINITY;
+#pragma unroll
+      for (int r = 0; r < ATTN_MAX_CLUSTER; ++r) {
+        if (r < cluster) {
+          const float2 ml = *cl.map_shared_rank(&blk_ml[n], r);
+          ms[r] = ml.x; ls[r] = ml.y;
+          os[r] = *cl.map_shared_rank(&blk_o[n][dd], r);
+          M = fmaxf(M, ml.x);
+        }
+      }
+      float L = 0.f, a = 0.f;
+#pragma unroll
+      for (int r = 0; r < ATTN_MAX_CLUSTER; ++r) {
+        if (r < cluster) {
+          const float sc = (ms[r] == -INFINITY) ? 0.f : exp2f(ms[r] - M);
+          L += ls[r] * sc;
+          a += os[r] * sc;
+        }
+      }
+      if (n_groups == 1) {
+        if (n < n_rows) {
+          const int tq = n / G, hh = n - tq * G;
+          const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+          out[row * DD_D + dd] = __float2bfloat16_rn(L > 0.f ? a / L : 0.f);
+          if (out_lse && dd == 0) out_lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+        }
+      } else {
+        part_o[((bg * n_groups + group) * ATTN_ROWS + n) * DD_D + dd] = a;
+        if (dd == 0) part_ml[(bg * n_groups + group) * ATTN_ROWS + n] = make_float2(M, L);
+      }
+    }
+    if (n_groups > 1) __threadfence();
+    cl.sync();                                   // nobody leaves while its shared memory may still be read
+    DD_TRACE_MARK(4);
+    if (n_groups == 1 || rank != 0) return;
+  } else {
+    // ---- one block per cluster: publish the block's partial directly
+    float* po = part_o + ((bg * n_groups + group) * ATTN_ROWS) * DD_D;
 #pragma unroll
     for (int n = 0; n < ATTN_ROWS; ++n) po[n * DD_D + d] = ob[n];
-    if (d < ATTN_ROWS) part_ml[(bg * n_splits + split) * ATTN_ROWS + d] = sm_ml[0][d];
+    if (d < ATTN_ROWS) part_ml[(bg * n_groups + group) * ATTN_ROWS + d] = blk_ml[d];
+    __threadfence();
+    __syncthreads();
   }
-  __threadfence();
-  __syncthreads();
+
+  // ---- several clusters: the last one to arrive merges the partials
   if (threadIdx.x == 0) {
     const unsigned prev = atomicAdd(&ticket[bg], 1u);
-    sm_last = (prev == (unsigned)(n_splits - 1));
+    sm_last = (prev == (unsigned)(n_groups - 1));
   }
   __syncthreads();
   if (!sm_last) return;
   __threadfence();
   if (threadIdx.x == 0) ticket[bg] = 0u;         // ready for the next launch
-#pragma unroll 1
-  for (int n = 0; n < n_rows; ++n) {
-    const float2* pml = part_ml + bg * n_splits * ATTN_ROWS + n;
+  // scale of every (group, row) and the row sums: warp w takes rows w and w+4, lanes take groups
+  float2* sm_lm = &sm_ml[0][0];                  // reused: [row] -> (max, sum)
+  float* sm_sc = &sm_o[0][0][0];                 // reused: [group][row] scale, n_groups <= ATTN_MAX_SPLITS
+  for (int n = warp; n < ATTN_ROWS; n += ATTN_WARPS) {
+    const float2* pml = part_ml + bg * n_groups * ATTN_ROWS + n;
+    float ms[ATTN_MAX_SPLITS / 32], ls[ATTN_MAX_SPLITS / 32];
     float M = -INFINITY;
-    for (int s = 0; s < n_splits; ++s) M = fmaxf(M, __ldcg(&pml[s * ATTN_ROWS].x));
-    float L = 0.f, a = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-      const float ms = __ldcg(&pml[s * ATTN_ROWS].x);
-      const float sc = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
-      L += __ldcg(&pml[s * ATTN_ROWS].y) * sc;
-      a += __ldcg(part_o + ((bg * n_splits + s) * ATTN_ROWS + n) * DD_D + d) * sc;
+#pragma unroll
+    for (int i = 0; i < ATTN_MAX_SPLITS / 32; ++i) {
+      const int sp = lane + 32 * i;
+      ms[i] = sp < n_groups ? __ldcg(&pml[sp * ATTN_ROWS].x) : -INFINITY;
+      ls[i] = sp < n_groups ? __ldcg(&pml[sp * ATTN_ROWS].y) : 0.f;
+      M = fmaxf(M, ms[i]);
     }
-    const int tq = n / G, hh = n - tq * G;
-    const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
-    out[row * DD_D + d] = __float2bfloat16_rn(L > 0.f ? a / L : 0.f);
-    if (out_lse && d == 0) out_lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    float L = 0.f;
+#pragma unroll
+    for (int i = 0; i < ATTN_MAX_SPLITS / 32; ++i) {
+      const int sp = lane + 32 * i;
+      const float sc = (ms[i] == -INFINITY) ? 0.f : exp2f(ms[i] - M);
+      if (sp < n_groups) sm_sc[sp * ATTN_ROWS + n] = sc;
+      L += ls[i] * sc;
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+    if (lane == 0) sm_lm[n] = make_float2(M, L);
   }
+  __syncthreads();
+  // every thread owns one channel of all rows; the loads of a group are independent of each other
+  float a[ATTN_ROWS];
+#pragma unroll
+  for (int n = 0; n < ATTN_ROWS; ++n) a[n] = 0.f;
+  const float* po = part_o + bg * n_groups * ATTN_ROWS * DD_D + d;
+#pragma unroll 4
+  for (int sp = 0; sp < n_groups; ++sp) {
+#pragma unroll
+    for (int n = 0; n < ATTN_ROWS; ++n) a[n] += __ldcg(po + (sp * ATTN_ROWS + n) * DD_D) * sm_sc[sp * ATTN_ROWS + n];
+  }
+#pragma unroll
+  for (int n = 0; n < ATTN_ROWS; ++n) {
+    if (n < n_rows) {
+      const float2 ml = sm_lm[n];
+      const int tq = n / G, hh = n - tq * G;
+      const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+      out[row * DD_D + d] = __float2bfloat16_rn(ml.y > 0.f ? a[n] / ml.y : 0.f);
+      if (out_lse && d == 0) out_lse[row] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
+    }
+  }
+}
+
+// Launch with clusters of `cluster` blocks along x (1 = no cluster attribute needed).
+static cudaError_t dd_attn_launch_raw(cudaStream_t st, int batch, int Hkv, int G, int Tq, int k, int n_splits,
+                                      int cluster, const void* q, const char* slot, const int* idx, const int* ctx_len,
+                                      void* out, float* out_lse, float* part_o, float2* part_ml, unsigned int* ticket) {
+  const int pps = (k + n_splits - 1) / n_splits;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_splits, Hkv, batch);
+  cfg.blockDim = dim3(ATTN_THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = cluster > 1 ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, dd_attn_kernel, (const __nv_bfloat16*)q, slot, idx, ctx_len, (__nv_bfloat16*)out,
+                            out_lse, part_o, part_ml, ticket, Hkv, G, Tq, k, n_splits, pps, cluster);
 }
 
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
                    float* out_lse, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
-  const int S = ctx->attn_splits;
-  const int pps = (c.k_pages + S - 1) / S;
-  dim3 grid(S, c.n_kv_heads, c.batch);
-  dd_attn_kernel<<<grid, ATTN_THREADS, 0, st>>>((const __nv_bfloat16*)q, slot, idx, ctx_len, (__nv_bfloat16*)out,
-                                                out_lse, ctx->attn_part_o, ctx->attn_part_ml, ctx->attn_ticket,
-                                                c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, S, pps);
-  DD_CUDA_TRY(ctx, cudaGetLastError());
+  DD_CUDA_TRY(ctx, dd_attn_launch_raw(st, c.batch, c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, ctx->attn_splits,
+                                      ctx->attn_cluster, q, slot, idx, ctx_len, out, out_lse, ctx->attn_part_o,
+                                      ctx->attn_part_ml, ctx->attn_ticket));
   return DD_OK;
 }
 
@@ -300,8 +453,8 @@ extern "C" int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_h
   if (batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads || k_pages < 1 || n_q_tokens < 1 ||
       n_q_tokens > 2 || n_q_tokens * (n_q_heads / n_kv_heads) > ATTN_ROWS)
     return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: unsupported geometry");
-  if (n_splits < 1 || n_splits > k_pages)
-    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: need 1 <= n_splits <= k_pages");
+  if (n_splits < 1 || n_splits > k_pages || n_splits > ATTN_MAX_SPLITS)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: need 1 <= n_splits <= min(k_pages, 64)");
   if (!q || !slot || !idx || !ctx_len || !out)
     return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: NULL tensor");
   if ((((uintptr_t)q) | ((uintptr_t)slot) | ((uintptr_t)out)) & 15)
@@ -336,13 +489,8 @@ extern "C" int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_h
   // the array keeps whatever the previous call (or an interrupted one) left: the arrival counters must start at zero
   e = cudaMemsetAsync(ticket, 0, (size_t)batch * n_kv_heads * sizeof(unsigned int), st);
   if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-  const int pps = (k_pages + n_splits - 1) / n_splits;
-  dim3 grid(n_splits, n_kv_heads, batch);
-  dd_attn_kernel<<<grid, ATTN_THREADS, 0, st>>>((const __nv_bfloat16*)q, (const char*)slot, idx, ctx_len,
-                                                (__nv_bfloat16*)out, out_lse, (float*)base, (float2*)(base + off_ml),
-                                                ticket, n_kv_heads, n_q_heads / n_kv_heads, n_q_tokens, k_pages,
-                                                n_splits, pps);
-  e = cudaGetLastError();
+  e = dd_attn_launch_raw(st, batch, n_kv_heads, n_q_heads / n_kv_heads, n_q_tokens, k_pages, n_splits, 1, q,
+                         (const char*)slot, idx, ctx_len, out, out_lse, (float*)base, (float2*)(base + off_ml), ticket);
   if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "dd_attn_kernel launch: %s", cudaGetErrorString(e));
   return DD_OK;
 }

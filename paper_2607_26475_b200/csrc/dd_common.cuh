@@ -23,7 +23,8 @@ struct dd_ctx {
   int G;                 // query heads per KV head
   int n_rows;            // Tq * G query rows that share one KV head
   int score_tiles;       // ceil(P / DD_SCORE_TILE)
-  int attn_splits;       // resolved split count
+  int attn_splits;       // resolved blocks per (request, KV head)
+  int attn_cluster;      // blocks per thread-block cluster (divides attn_splits)
   size_t slot_bytes;
   // scratch (device)
   float* score_s;        // [B][Hkv][P][G] scaled logits

@@ -144,26 +144,35 @@ def test_invalid_configurations_are_rejected(dd):
         assert e.value.code == dd.DD_ERR_INVALID_ARG
 
 
-def test_config2_launch_configuration_sampled(dd):
-    """Config 2 as the benchmark launches it (L=32, B=8, 32768-token contexts, 2048 of them selected per KV
-    head, ring depth 2). The host store aliases two physical layers to stay small; sampled (step, layer,
-    request) outputs are checked one by one against the oracle."""
-    w = wl.CONFIGS[2]
-    L, B, P, k, S, n_phys = w.n_layers, w.batch, w.n_pages, w.k_pages, 2, 2
+@pytest.mark.parametrize("cfg,n_phys,samples", [
+    (2, 2, [(0, 0, 0), (0, 17, 7), (1, 31, 3), (1, 16, 0)]),
+    (3, 1, [(0, 5, 31), (1, 30, 0)]),
+    (4, 1, [(0, 0, 7), (1, 31, 2)]),
+    (5, 1, [(0, 3, 0), (1, 28, 0)]),
+])
+def test_full_launch_configuration_sampled(dd, cfg, n_phys, samples):
+    """Configs 2-5 as the benchmark launches them (32 layers, full batch, full context and budget, ring depth
+    2). The host store aliases `n_phys` physical layers to stay small; sampled (step, layer, request)
+    outputs are checked one by one against the oracle."""
+    w = wl.CONFIGS[cfg]
+    L, B, P, k, S, F = w.n_layers, w.batch, w.n_pages, w.k_pages, 2, w.forced_recent_pages
     ctx_len = wl.ctx_lens(w)
     npg = torch.full((B,), P, dtype=torch.int32)
-    c = dd.Context(n_layers=L, batch=B, max_pages=P, k_pages=k)
+    c = dd.Context(n_layers=L, batch=B, max_pages=P, k_pages=k, forced_recent_pages=F)
+    one = dd.Context(n_layers=1, batch=1, max_pages=P, k_pages=1)
     phys, lms = [], []
     for l in range(n_phys):
-        dev = torch.stack([wl.kv_slab(w, l, b, device="cuda") for b in range(B)])
+        host = torch.empty((B, HKV, P, 2, T, D), dtype=torch.bfloat16, pin_memory=True)
         lm = torch.empty((B, HKV, P, D), dtype=torch.bfloat16, device="cuda")
-        c.build_landmarks(dev, ctx_len.cuda(), lm)
-        host = torch.empty(dev.shape, dtype=torch.bfloat16, pin_memory=True)
-        host.copy_(dev)
+        for b in range(B):
+            dev = wl.kv_slab(w, l, b, device="cuda")
+            one.build_landmarks(dev, ctx_len[b:b + 1].cuda(), lm[b])
+            host[b].copy_(dev)
+            del dev
         phys.append(host)
         lms.append(lm)
-        del dev
     torch.cuda.synchronize()
+    one.close()
     store = [phys[l % n_phys] for l in range(L)]
     lm_l = [lms[l % n_phys] for l in range(L)]
     q_init = torch.stack([wl.queries(w, -1, l)[:, 1] for l in range(L)])
@@ -180,18 +189,19 @@ def test_config2_launch_configuration_sampled(dd):
     c.sync()
     assert c.device_error() == (0, 0)
     n_exact = n_all = 0
-    for t, l, b in [(0, 0, 0), (0, 17, 7), (1, 31, 3), (1, 16, 0)]:
-        kv_b = f32(store[l][b:b + 1])
-        lm_want = orc.build_landmarks(kv_b[:, :, :, 0], ctx_len[b:b + 1].numpy())
+    for t, l, b in samples:
+        kv_b = store[l][b:b + 1]
+        lm_want = orc.build_landmarks(f32(kv_b[:, :, :, 0]), ctx_len[b:b + 1].numpy())
         assert np.array_equal(f32(lm_l[l][b:b + 1]), lm_want), "device-built landmarks differ from the oracle's"
         qsel = f32(q_init[l][b:b + 1]) if t == 0 else f32(q_steps[t - 1, l][b:b + 1, 1])
-        _, sc = orc.select_topk(qsel, lm_want, npg[b:b + 1].numpy(), k)
+        _, sc = orc.select_topk(qsel, lm_want, npg[b:b + 1].numpy(), k, F)
         got = idxs[t][l][b:b + 1]
         for h in range(HKV):
-            n_exact += check_selection(got[0, h], sc[0][h], k, 0)
+            n_exact += check_selection(got[0, h], sc[0][h], k, F)
             n_all += 1
-        slot = orc.gather_kv(kv_b, got)
+        slot_bits = orc.gather_kv(raw16(kv_b), got)                     # bit copy of the selected pages only
+        slot = (slot_bits.astype(np.uint32) << 16).view(np.float32)
         want, _ = orc.sparse_decode_attn(f32(q_steps[t, l][b:b + 1]), slot, got, ctx_len[b:b + 1].numpy(), T)
         check_attention(outs[t, l][b:b + 1], want)
-    print(f"exact index sets: {n_exact}/{n_all}")
+    print(f"config {cfg}: exact index sets {n_exact}/{n_all}")
     c.close()

@@ -47,10 +47,10 @@ def test_static_entry_point_matches_the_context_entry_point_on_consecutive_calls
     from paper_2607_26475_b200 import binding as dd
     assert dd.lib.dd_static_scratch_capacity() == 8 << 20
     # two calls in a row with different shapes and split counts: the second finds the first one's leftovers
-    e1 = _case(dd, 1, B=3, P=200, k=64, splits_ctx=4, splits_static=4, ctx_len=[3200, 3190, 1700])
+    e1 = _case(dd, 1, B=3, P=200, k=64, splits_ctx=5, splits_static=5, ctx_len=[3200, 3190, 1700])
     e2 = _case(dd, 2, B=2, P=150, k=37, splits_ctx=1, splits_static=5, ctx_len=[2400, 2399])
-    e3 = _case(dd, 3, B=3, P=200, k=64, splits_ctx=4, splits_static=4, ctx_len=[3200, 3190, 1700])
-    assert e1 == 0.0 and e3 == 0.0          # same split geometry gives the same bits as the context path
+    e3 = _case(dd, 3, B=3, P=200, k=64, splits_ctx=5, splits_static=5, ctx_len=[3200, 3190, 1700])
+    assert e1 == 0.0 and e3 == 0.0          # same split geometry (no clusters) gives the same bits as the context path
     assert e2 <= ATTN_MAX_ABS
 
 
