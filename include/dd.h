@@ -49,6 +49,9 @@ extern "C" {
 #define DD_GATHER_LOADS  0          /* zero-copy: warps read the pinned pages with 16-byte loads */
 #define DD_GATHER_BULK   1          /* bulk-copy engine: pinned page -> shared memory -> slot (cp.async.bulk) */
 
+#define DD_SELECT_AUTO         0    /* fused cluster kernel when the request fits, else the two-kernel path */
+#define DD_SELECT_TWO_KERNELS  1    /* scoring kernel + top-k kernel with logits in global scratch */
+
 typedef struct dd_ctx dd_ctx;
 
 typedef struct dd_config {
@@ -65,6 +68,7 @@ typedef struct dd_config {
   int ring_depth;            /* D >= 2 (2 = the two-buffer scheme) */
   int gather_mode;           /* DD_GATHER_LOADS or DD_GATHER_BULK */
   int gather_ctas;           /* thread blocks the gather may occupy; 0 = library default */
+  int select_mode;           /* DD_SELECT_AUTO or DD_SELECT_TWO_KERNELS */
   int attn_splits;           /* blocks per (request, KV head) in attention, <= 64 or a multiple of 8 up to 512; 0 = automatic */
   void* compute_stream;      /* cudaStream_t used by the pipelined calls for attention and selection */
   void* copy_stream;         /* cudaStream_t used by the pipelined calls for the gather */

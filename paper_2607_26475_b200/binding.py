@@ -25,6 +25,8 @@ DD_ERR_STATE = -6
 DD_ERR_WAIT_EXPIRED = -7
 DD_GATHER_LOADS = 0
 DD_GATHER_BULK = 1
+DD_SELECT_AUTO = 0
+DD_SELECT_TWO_KERNELS = 1
 
 EXPORTS = [
     "dd_create", "dd_destroy", "dd_slot_bytes", "dd_ring_bytes", "dd_scratch_bytes", "dd_slot_ptr",
@@ -40,7 +42,7 @@ class DDConfig(C.Structure):
         ("n_layers", C.c_int), ("batch", C.c_int), ("n_q_heads", C.c_int), ("n_kv_heads", C.c_int),
         ("head_dim", C.c_int), ("page_tokens", C.c_int), ("max_pages", C.c_int), ("k_pages", C.c_int),
         ("forced_recent_pages", C.c_int), ("n_q_tokens", C.c_int), ("ring_depth", C.c_int),
-        ("gather_mode", C.c_int), ("gather_ctas", C.c_int), ("attn_splits", C.c_int),
+        ("gather_mode", C.c_int), ("gather_ctas", C.c_int), ("select_mode", C.c_int), ("attn_splits", C.c_int),
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
     ]
@@ -136,14 +138,14 @@ class Context:
 
     def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
-                 gather_ctas=0, attn_splits=0, compute_stream=None, copy_stream=None, ring=None):
+                 gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
         self.copy_stream = copy_stream if copy_stream is not None else torch.cuda.Stream()
         self._ring = ring
         self.cfg = DDConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, page_tokens, max_pages, k_pages,
-                            forced_recent_pages, n_q_tokens, ring_depth, gather_mode, gather_ctas, attn_splits,
+                            forced_recent_pages, n_q_tokens, ring_depth, gather_mode, gather_ctas, select_mode, attn_splits,
                             self.compute_stream.cuda_stream, self.copy_stream.cuda_stream,
                             _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0)
         self._h = C.c_void_p()

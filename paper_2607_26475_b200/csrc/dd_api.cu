@@ -56,6 +56,7 @@ static const char* dd_check_config(const dd_config* c) {
   if (c->forced_recent_pages < 0 || c->forced_recent_pages > c->k_pages) return "need 0 <= forced_recent_pages <= k_pages";
   if (c->ring_depth < 2 || c->ring_depth > DD_MAX_RING) return "ring_depth must be in [2, 8]";
   if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK) return "unknown gather_mode";
+  if (c->select_mode != DD_SELECT_AUTO && c->select_mode != DD_SELECT_TWO_KERNELS) return "unknown select_mode";
   if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
   if (c->attn_splits > 512) return "attn_splits must be <= 512";
   if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";

@@ -18,24 +18,8 @@
 
 #include "dd_common.cuh"
 
-// Optional per-block timeline for tuning (compile with -DDD_TRACE; never in the shipped library):
-// mark i of block (x, y, z) is the global nanosecond timer when thread 0 passed it.
-#ifdef DD_TRACE
-__device__ unsigned long long dd_trace_buf[1 << 16][8];
-#define DD_TRACE_MARK(i)                                                                                     \
-  do {                                                                                                       \
-    if (threadIdx.x == 0) {                                                                                  \
-      unsigned long long t__;                                                                                \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));                                                \
-      dd_trace_buf[(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x][i] = t__;                 \
-    }                                                                                                        \
-  } while (0)
-extern "C" int dd_trace_read(unsigned long long* host, size_t bytes) {
-  return (int)cudaMemcpyFromSymbol(host, dd_trace_buf, bytes);
-}
-#else
-#define DD_TRACE_MARK(i)
-#endif
+DD_TRACE_DECLARE(dd_trace_attn)
+#define DD_TRACE_MARK(i) DD_TRACE_MARK_IN(dd_trace_attn, i)
 
 constexpr int ATTN_WARPS = 4;
 constexpr int ATTN_THREADS = ATTN_WARPS * 32;

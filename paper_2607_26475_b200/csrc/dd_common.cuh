@@ -25,6 +25,9 @@ struct dd_ctx {
   int score_tiles;       // ceil(P / DD_SCORE_TILE)
   int attn_splits;       // resolved blocks per (request, KV head)
   int attn_cluster;      // blocks per thread-block cluster (divides attn_splits)
+  int sel_cluster;       // blocks per cluster of the fused selection kernel; 0 = two-kernel path
+  int sel_ppc;           // pages per block of the fused selection
+  int sel_smem_bytes;
   size_t slot_bytes;
   // scratch (device)
   float* score_s;        // [B][Hkv][P][G] scaled logits
@@ -110,5 +113,26 @@ __device__ __forceinline__ void dd_ml_merge(float& m, float& l, float m2, float 
   l = l * a + l2 * b;
   m = mn;
 }
+
+// Optional per-block timeline for tuning (compile with -DDD_TRACE; never in the shipped library): mark i of
+// block (x, y, z) is the global nanosecond timer when thread 0 passed it; <name>_read copies the table out.
+#ifdef DD_TRACE
+#define DD_TRACE_DECLARE(name)                                                                       \
+  __device__ unsigned long long name[1 << 16][8];                                                    \
+  extern "C" int name##_read(unsigned long long* host, size_t bytes) {                               \
+    return (int)cudaMemcpyFromSymbol(host, name, bytes);                                             \
+  }
+#define DD_TRACE_MARK_IN(name, i)                                                                    \
+  do {                                                                                               \
+    if (threadIdx.x == 0) {                                                                          \
+      unsigned long long t__;                                                                        \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));                                        \
+      name[(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x][i] = t__;                 \
+    }                                                                                                \
+  } while (0)
+#else
+#define DD_TRACE_DECLARE(name)
+#define DD_TRACE_MARK_IN(name, i)
+#endif
 
 #endif  // __CUDACC__

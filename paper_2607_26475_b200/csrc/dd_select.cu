@@ -5,6 +5,8 @@
 // kernel turns the per-head logits into log-probabilities with the per-head log-sum-exp, takes the
 // group maximum, and finds the k-th largest by an MSB-first radix select on order-preserving keys,
 // followed by an ordered compaction that emits ascending page numbers.
+#include <cooperative_groups.h>
+
 #include "dd_common.cuh"
 
 // ------------------------------------------------------------------------------------------------
@@ -282,16 +284,17 @@ __global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
     const uint32_t kmin = sh_min;
     const uint32_t range = sh_max - kmin;
     const int nbits = 32 - __clz(range);
-    const int passes = (nbits + RADIX_BITS - 1) / RADIX_BITS;
     unsigned long long prefix = 0;
     k_rem = (unsigned)k_free;
-    for (int pass = 0; pass < passes; ++pass) {
-      const int shift = (passes - 1 - pass) * RADIX_BITS;
+    int hi = nbits;                              // unresolved bits of (key - min); digits are cut from the top
+    while (hi > 0) {
+      const int width = hi < RADIX_BITS ? hi : RADIX_BITS;
+      const int shift = hi - width;
       for (int i = tid; i < RADIX_BINS; i += TOPK_THREADS) hist[i] = 0u;
       __syncthreads();
       for (int p = tid; p < n_free; p += TOPK_THREADS) {
         const unsigned long long rel = (unsigned long long)(keys[p] - kmin);
-        if ((rel >> (shift + RADIX_BITS)) == prefix) atomicAdd(&hist[(unsigned)(rel >> shift) & (RADIX_BINS - 1)], 1u);
+        if ((rel >> hi) == prefix) atomicAdd(&hist[(unsigned)(rel >> shift) & ((1u << width) - 1u)], 1u);
       }
       __syncthreads();
       // thread i owns bins 2047-2i and 2046-2i; scan from the top bin downwards
@@ -303,8 +306,9 @@ __global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
         else { sh_bin = RADIX_BINS - 2 - 2 * tid; sh_above = above + h_hi; }
       }
       __syncthreads();
-      prefix = (prefix << RADIX_BITS) | sh_bin;
+      prefix = (prefix << width) | sh_bin;
       k_rem -= sh_above;
+      hi = shift;
       __syncthreads();
     }
     thr = kmin + (uint32_t)prefix;               // k_rem of the keys equal to thr are still to be taken
@@ -334,10 +338,378 @@ __global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
   for (int j = k_eff + tid; j < k; j += TOPK_THREADS) out[j] = np > 0 ? np - 1 : 0;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Fused selection: one thread-block cluster per (request, KV head).
+//
+// Block `rank` of the cluster scores the pages [rank*ppc, (rank+1)*ppc) and keeps their logits in its own
+// shared memory; what the blocks must agree on travels through distributed shared memory:
+//   1. per-head (max, sum exp) of every block      -> log-sum-exp of the request
+//   2. min / max of the order-preserving keys      -> digit positions of the radix select
+//   3. per radix pass, the sums of 8-bin groups and the 8 bins of one group; then the few keys that share
+//      the leading digits                          -> the k-th largest key (every block derives it)
+//   4. per-block counts of selected pages          -> where each block's pages go in the ascending output
+// Nothing but the landmarks is read from global memory, and nothing but the index set is written.
+// ------------------------------------------------------------------------------------------------
+namespace cg = cooperative_groups;
+
+DD_TRACE_DECLARE(dd_trace_select)
+#define DD_SEL_MARK(i) DD_TRACE_MARK_IN(dd_trace_select, i)
+
+constexpr int SEL_THREADS = 256;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int SEL_CAND_MAX = 512;          // keys sharing a radix prefix that are ranked directly
+constexpr int SEL_MAX_SMEM = 200 * 1024;   // dynamic shared memory the fused kernel may be launched with
+
+// Exclusive prefix sum over the 256 threads of the block; `total` is returned to every thread.
+__device__ __forceinline__ unsigned dd_scan256_excl(unsigned v, unsigned* warp_tot, unsigned& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned inc = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, inc, off);
+    if (lane >= off) inc += n;
+  }
+  __syncthreads();
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  const unsigned wt = lane < SEL_WARPS ? warp_tot[lane] : 0u;
+  unsigned winc = wt;
+#pragma unroll
+  for (int off = 1; off < SEL_WARPS; off <<= 1) {
+    const unsigned n = __shfl_up_sync(0xffffffffu, winc, off);
+    if (lane >= off) winc += n;
+  }
+  total = __shfl_sync(0xffffffffu, winc, SEL_WARPS - 1);
+  const unsigned wexcl = __shfl_sync(0xffffffffu, winc - wt, warp);
+  return wexcl + inc - v;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
+    const __nv_bfloat16* __restrict__ q, int q_req_stride, int q_token_off, const __nv_bfloat16* __restrict__ lm,
+    const int* __restrict__ n_pages, int* __restrict__ out_idx, float* __restrict__ out_scores, int P, int G, int Hkv,
+    int k, int forced, int ppc, int* err_word) {
+  extern __shared__ __align__(16) unsigned char sel_smem[];
+  float* s_sm = reinterpret_cast<float*>(sel_smem);                              // [ppc][G] logits; key in [p][0]
+  unsigned* hist = reinterpret_cast<unsigned*>(sel_smem + (size_t)ppc * G * 4);  // [2][RADIX_BINS]
+  __shared__ float2 cta_ml[8];
+  __shared__ unsigned cta_minmax[2];
+  __shared__ unsigned cta_cnt[2];
+  __shared__ float2 red[SEL_WARPS][8];
+  __shared__ float lse_s[8];
+  __shared__ unsigned warp_tot[SEL_WARPS];
+  __shared__ unsigned sh_bin, sh_above, sh_grp, sh_cnt, sh_thr, cand_n;
+  __shared__ unsigned grp[2][SEL_THREADS];
+  __shared__ unsigned cnt8[8];
+  __shared__ uint32_t cand[SEL_CAND_MAX];
+  __shared__ uint32_t all_c[SEL_CAND_MAX];
+
+  cg::cluster_group cl = cg::this_cluster();
+  const int C = (int)cl.num_blocks();
+  const int rank = (int)cl.block_rank();
+  const int g = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const size_t bg = (size_t)b * Hkv + g;
+  int np = n_pages[b];
+  if (np > P || np < k) {
+    if (tid == 0 && rank == 0) dd_report(err_word, DD_ERR_INDEX_RANGE, np);
+    np = np > P ? P : (np < 0 ? 0 : np);
+  }
+  const int k_eff = k < np ? k : np;
+  const int forced_eff = forced < k_eff ? forced : k_eff;
+  const int n_free = np - forced_eff;            // pages [n_free, np) are forced
+  const int k_free = k_eff - forced_eff;
+  const int p_lo = rank * ppc;
+  const int n_local = max(0, min(np, p_lo + ppc) - p_lo);
+  if (tid == 0) { cta_minmax[0] = 0xFFFFFFFFu; cta_minmax[1] = 0u; cta_cnt[0] = 0u; cta_cnt[1] = 0u; cand_n = 0u; }
+
+  DD_SEL_MARK(0);
+  // ---- A. logits of this block's pages (same MMA formulation as dd_score_kernel), kept in shared memory
+  float m_run[2] = {-INFINITY, -INFINITY};
+  float l_run[2] = {0.f, 0.f};
+  {
+    uint4 qf[4];
+    if (gl < G) {
+      const uint4* qrow = reinterpret_cast<const uint4*>(q + (size_t)b * q_req_stride + q_token_off +
+                                                         (size_t)(g * G + gl) * DD_D);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = __ldg(qrow + kk * 4 + t);
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * DD_D;
+    const float scale = rsqrtf((float)DD_D);
+    for (int t0 = warp * 32; t0 < n_local; t0 += SEL_WARPS * 32) {     // two 16-page MMA tiles per trip
+      uint4 lo[2][4], hi[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const int pa = min(p_lo + t0 + mt * 16 + gl, P - 1);           // stay inside the tensor; discarded later
+        const int pb = min(p_lo + t0 + mt * 16 + gl + 8, P - 1);
+        const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D);
+        const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          lo[mt][kk] = dd_ld_stream(ra + kk * 4 + t);
+          hi[mt][kk] = dd_ld_stream(rb + kk * 4 + t);
+        }
+      }
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          dd_mma_bf16(acc, lo[mt][kk].x, hi[mt][kk].x, lo[mt][kk].y, hi[mt][kk].y, qf[kk].x, qf[kk].y);
+          dd_mma_bf16(acc, lo[mt][kk].z, hi[mt][kk].z, lo[mt][kk].w, hi[mt][kk].w, qf[kk].z, qf[kk].w);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int pl = t0 + mt * 16 + gl + r * 8;                     // page within the block
+          if (pl < n_local) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              const int h = 2 * t + c;
+              if (h < G) {
+                const float v = acc[2 * r + c] * scale;
+                s_sm[(size_t)pl * G + h] = v;
+                const float mn = fmaxf(m_run[c], v);
+                l_run[c] = l_run[c] * expf(m_run[c] - mn) + expf(v - mn);
+                m_run[c] = mn;
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+      const float m2 = __shfl_xor_sync(0xffffffffu, m_run[c], off);
+      const float l2 = __shfl_xor_sync(0xffffffffu, l_run[c], off);
+      dd_ml_merge(m_run[c], l_run[c], m2, l2, false);
+    }
+  }
+  if (gl == 0) {
+    red[warp][2 * t] = make_float2(m_run[0], l_run[0]);
+    red[warp][2 * t + 1] = make_float2(m_run[1], l_run[1]);
+  }
+  __syncthreads();
+  if (tid < 8) {
+    float m = red[0][tid].x, l = red[0][tid].y;
+#pragma unroll
+    for (int w = 1; w < SEL_WARPS; ++w) dd_ml_merge(m, l, red[w][tid].x, red[w][tid].y, false);
+    cta_ml[tid] = make_float2(m, l);
+  }
+  DD_SEL_MARK(1);
+  // ---- B. log-sum-exp of the whole request: every block merges the partials of all blocks
+  cl.sync();
+  DD_SEL_MARK(2);
+  if (tid < G) {
+    float m = -INFINITY, l = 0.f;
+    for (int r = 0; r < C; ++r) {
+      const float2 v = *cl.map_shared_rank(&cta_ml[tid], r);
+      dd_ml_merge(m, l, v.x, v.y, false);
+    }
+    lse_s[tid] = m + logf(l);
+  }
+  __syncthreads();
+
+  // ---- C. keys in place of the first logit of every page; block min / max of the non-forced keys
+  {
+    float lse[8];
+#pragma unroll
+    for (int h = 0; h < 8; ++h) lse[h] = h < G ? lse_s[h] : 0.f;
+    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+    for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
+      float c = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < 8; ++h)
+        if (h < G) c = fmaxf(c, s_sm[(size_t)pl * G + h] - lse[h]);
+      const int p = p_lo + pl;
+      if (out_scores) out_scores[bg * P + p] = expf(c);
+      uint32_t key = dd_orderable(c);
+      if (p >= n_free) key = 0xFFFFFFFFu;
+      else { kmin = min(kmin, key); kmax = max(kmax, key); }
+      reinterpret_cast<uint32_t*>(s_sm)[(size_t)pl * G] = key;
+    }
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { atomicMin(&cta_minmax[0], kmin); atomicMax(&cta_minmax[1], kmax); }
+  }
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(s_sm);      // key of local page pl at keys[pl * G]
+  DD_SEL_MARK(3);
+  cl.sync();
+  DD_SEL_MARK(4);
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+  for (int r = 0; r < C; ++r) {
+    kmin = min(kmin, *cl.map_shared_rank(&cta_minmax[0], r));
+    kmax = max(kmax, *cl.map_shared_rank(&cta_minmax[1], r));
+  }
+  const int n_free_local = max(0, min(n_free, p_lo + ppc) - p_lo);     // local pages that take part in the select
+
+  // ---- D. the k_free-th largest key. MSB-first radix passes on (key - min); a pass exchanges only the sums
+  // of 8-bin groups and then the 8 bins of the group where the count crosses k. As soon as the crossing bin
+  // holds few keys, those keys themselves are exchanged and ranked, which ends the search.
+  uint32_t thr = 0xFFFFFFFFu;
+  unsigned k_rem = 0;
+  if (k_free > 0) {
+    const uint32_t range = kmax - kmin;
+    const int nbits = 32 - __clz(range);
+    unsigned long long prefix = 0;
+    k_rem = (unsigned)k_free;
+    thr = kmin;                                   // all keys equal (nbits == 0): take the first k_free of them
+    bool done = false;
+    int hi = nbits;                               // bits of (key - min) not resolved yet; digits are cut from the top
+    for (int pass = 0; hi > 0 && !done; ++pass) {
+      const int width = hi < RADIX_BITS ? hi : RADIX_BITS;
+      const int shift = hi - width;
+      unsigned* h = hist + (pass & 1) * RADIX_BINS;                     // double-buffered: peers may still read the other
+      unsigned* gp = grp[pass & 1];
+      for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) h[i] = 0u;
+      __syncthreads();
+      for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
+        const unsigned long long rel = (unsigned long long)(keys[(size_t)pl * G] - kmin);
+        if ((rel >> hi) == prefix) atomicAdd(&h[(unsigned)(rel >> shift) & ((1u << width) - 1u)], 1u);
+      }
+      __syncthreads();
+      {                                           // thread i owns the 8 bins [2047-8i-7, 2047-8i]
+        unsigned sum8 = 0;
+#pragma unroll
+        for (int jb = 0; jb < 8; ++jb) sum8 += h[RADIX_BINS - 1 - 8 * tid - jb];
+        gp[tid] = sum8;
+      }
+      cl.sync();
+      unsigned tot = 0;
+      for (int r = 0; r < C; ++r) tot += cl.map_shared_rank(gp, r)[tid];
+      unsigned total;
+      const unsigned above = dd_scan256_excl(tot, warp_tot, total);      // groups are scanned from the top bin down
+      if (above < k_rem && k_rem <= above + tot) { sh_grp = (unsigned)tid; sh_above = above; }
+      __syncthreads();
+      const int gsel = (int)sh_grp;
+      if (tid < 8) {
+        unsigned c8 = 0;
+        for (int r = 0; r < C; ++r) c8 += cl.map_shared_rank(h, r)[RADIX_BINS - 1 - 8 * gsel - tid];
+        cnt8[tid] = c8;
+      }
+      __syncthreads();
+      if (tid == 0) {
+        unsigned ab = sh_above;
+        for (int jb = 0; jb < 8; ++jb) {
+          if (ab < k_rem && k_rem <= ab + cnt8[jb]) { sh_bin = RADIX_BINS - 1 - 8 * gsel - jb; sh_above = ab; sh_cnt = cnt8[jb]; break; }
+          ab += cnt8[jb];
+        }
+      }
+      __syncthreads();
+      prefix = (prefix << width) | sh_bin;
+      k_rem -= sh_above;                          // keys in higher bins are all selected
+      const unsigned bin_cnt = sh_cnt;
+      hi = shift;
+      __syncthreads();
+      if (hi == 0) {
+        thr = kmin + (uint32_t)prefix;            // k_rem of the keys equal to thr are still to be taken
+      } else if (bin_cnt <= (unsigned)SEL_CAND_MAX) {
+        // few keys share the prefix: every block lists its own, all blocks read all lists and rank them
+        for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
+          const uint32_t key = keys[(size_t)pl * G];
+          if (((unsigned long long)(key - kmin) >> shift) == prefix) cand[atomicAdd(&cand_n, 1u)] = key;
+        }
+        cl.sync();
+        unsigned off = 0;
+        for (int r = 0; r < C; ++r) {
+          const unsigned n_r = *cl.map_shared_rank(&cand_n, r);
+          const uint32_t* cr = cl.map_shared_rank(cand, r);
+          for (unsigned i = tid; i < n_r; i += SEL_THREADS) all_c[off + i] = cr[i];
+          off += n_r;
+        }
+        __syncthreads();
+        for (unsigned i = tid; i < off; i += SEL_THREADS) {
+          const uint32_t v = all_c[i];
+          unsigned gtc = 0, gec = 0;
+          for (unsigned j = 0; j < off; ++j) {
+            const uint32_t u = all_c[j];
+            gtc += u > v;
+            gec += u >= v;
+          }
+          if (gtc < k_rem && k_rem <= gec) { sh_thr = v; sh_above = gtc; }   // equal candidates write equal values
+        }
+        __syncthreads();
+        thr = sh_thr;
+        k_rem -= sh_above;
+        done = true;
+      }
+    }
+  }
+  DD_SEL_MARK(5);
+
+  // ---- E. how many pages each block contributes, then ordered compaction of this block's pages
+  {
+    unsigned gt = 0, eq = 0;
+    for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
+      const uint32_t key = keys[(size_t)pl * G];
+      if (p_lo + pl >= n_free || key > thr) ++gt;
+      else if (key == thr) ++eq;
+    }
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    eq = __reduce_add_sync(0xffffffffu, eq);
+    if (lane == 0) { atomicAdd(&cta_cnt[0], gt); atomicAdd(&cta_cnt[1], eq); }
+  }
+  cl.sync();
+  DD_SEL_MARK(6);
+  unsigned base_gt = 0, base_eq = 0;
+  for (int r = 0; r < rank; ++r) {
+    base_gt += *cl.map_shared_rank(&cta_cnt[0], r);
+    base_eq += *cl.map_shared_rank(&cta_cnt[1], r);
+  }
+  int* out = out_idx + bg * k;
+  for (int c0 = 0; c0 < n_local; c0 += SEL_THREADS) {
+    const int pl = c0 + tid;
+    unsigned gt = 0, eq = 0;
+    if (pl < n_local) {
+      const uint32_t key = keys[(size_t)pl * G];
+      if (p_lo + pl >= n_free || key > thr) gt = 1;
+      else if (key == thr) eq = 1;
+    }
+    unsigned total;
+    const unsigned ex = dd_scan256_excl(gt | (eq << 16), warp_tot, total);
+    const unsigned eq_before = base_eq + (ex >> 16);
+    if (gt || (eq && eq_before < k_rem)) {
+      const unsigned pos = base_gt + (ex & 0xFFFFu) + min(eq_before, k_rem);
+      if (pos < (unsigned)k) out[pos] = p_lo + pl;
+    }
+    base_gt += total & 0xFFFFu;
+    base_eq += total >> 16;
+  }
+  if (rank == 0)                                 // precondition k <= n_pages violated: pad with the last valid page
+    for (int j = k_eff + tid; j < k; j += SEL_THREADS) out[j] = np > 0 ? np - 1 : 0;
+  cl.sync();                                     // nobody leaves while its shared memory may still be read
+  DD_SEL_MARK(7);
+}
+
 int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
                      const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
   const int G = ctx->G;
+  if (ctx->sel_cluster > 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ctx->sel_cluster, c.n_kv_heads, c.batch);
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.dynamicSmemBytes = ctx->sel_smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = ctx->sel_cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    DD_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, dd_select_fused_kernel, (const __nv_bfloat16*)q,
+                                        q_tokens_in_tensor * c.n_q_heads * DD_D, q_token * c.n_q_heads * DD_D,
+                                        (const __nv_bfloat16*)landmarks, n_pages, out_idx, out_scores, c.max_pages, G,
+                                        c.n_kv_heads, c.k_pages, c.forced_recent_pages, ctx->sel_ppc, ctx->err_word));
+    return DD_OK;
+  }
   dim3 sgrid(ctx->score_tiles, c.n_kv_heads, c.batch);
   dd_score_kernel<<<sgrid, 128, 0, st>>>((const __nv_bfloat16*)q, q_tokens_in_tensor * c.n_q_heads * DD_D,
                                          q_token * c.n_q_heads * DD_D, (const __nv_bfloat16*)landmarks, n_pages,
@@ -352,8 +724,56 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
   return DD_OK;
 }
 
+// Picks the cluster size of the fused selection: a power of two such that all clusters are resident at once
+// (two blocks per SM), every block has at least 32 pages, and a block's share of the logits fits in shared
+// memory. Up to 8 blocks, 16 for very long requests. 0 = not possible, use the two-kernel path.
+static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
+  const dd_config& c = ctx->cfg;
+  const int G = ctx->G;
+  const int problems = c.batch * c.n_kv_heads;
+  // function attributes are per process, not per context: always ask for the largest the kernel may use
+  if (cudaFuncSetAttribute(dd_select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEL_MAX_SMEM) !=
+      cudaSuccess) { cudaGetLastError(); return 0; }
+  const bool big_ok = cudaFuncSetAttribute(dd_select_fused_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
+                                           1) == cudaSuccess;
+  if (!big_ok) cudaGetLastError();
+  const int c_max = (c.max_pages >= 32768 && big_ok) ? 16 : 8;
+  int C = 1;
+  while (C * 2 <= c_max && C * 2 * problems <= 2 * ctx->sm_count && c.max_pages / (C * 2) >= 32) C *= 2;
+  for (; C <= c_max; C *= 2) {
+    int ppc = (c.max_pages + C - 1) / C;
+    ppc = (ppc + 31) & ~31;                                // whole pairs of MMA tiles
+    const size_t smem = (size_t)ppc * G * 4 + 2 * RADIX_BINS * 4;
+    if (smem > (size_t)SEL_MAX_SMEM) continue;             // too long for this cluster size: try a larger one
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(C, c.n_kv_heads, c.batch);
+    cfg.blockDim = dim3(SEL_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, dd_select_fused_kernel, &cfg) != cudaSuccess || n_clusters < 1) {
+      cudaGetLastError();
+      if (C == 16) { C = 4; continue; }                    // 16-block clusters unavailable: fall back to 8
+      continue;
+    }
+    *ppc_out = ppc;
+    *smem_out = (int)smem;
+    return C;
+  }
+  return 0;
+}
+
 int dd_select_setup(dd_ctx* ctx) {
   DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(TOPK_SMEM_KEYS * sizeof(uint32_t))));
+  ctx->sel_cluster = 0;
+  if (ctx->cfg.select_mode != DD_SELECT_TWO_KERNELS)
+    ctx->sel_cluster = dd_select_pick_cluster(ctx, &ctx->sel_ppc, &ctx->sel_smem_bytes);
   return DD_OK;
 }

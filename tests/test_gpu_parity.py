@@ -29,14 +29,14 @@ def _layer_store(w, layer, pinned=True):
     return kv.pin_memory() if pinned else kv
 
 
-def _select_case(dd, B, P, k, forced, n_pages, seed, G=4, Tq=2, scale=1.0):
+def _select_case(dd, B, P, k, forced, n_pages, seed, G=4, Tq=2, scale=1.0, select_mode=0):
     Hq = HKV * G
     g = torch.Generator().manual_seed(seed)
     lm = torch.randn(B, HKV, P, D, generator=g).mul(scale).to(torch.bfloat16)
     q = torch.randn(B, Tq, Hq, D, generator=g).to(torch.bfloat16)
     npg = torch.tensor(n_pages, dtype=torch.int32)
     ctx = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_kv_heads=HKV,
-                     forced_recent_pages=forced, n_q_tokens=Tq)
+                     forced_recent_pages=forced, n_q_tokens=Tq, select_mode=select_mode)
     idx = torch.full((B, HKV, k), -7, dtype=torch.int32, device="cuda")
     scores = torch.full((B, HKV, P), -1.0, dtype=torch.float32, device="cuda")
     qt = Tq - 1
@@ -98,22 +98,29 @@ def test_select_config1_shape_needles(dd):
     (2, 517, 16, 0, [517, 300], 1, 2),             # G = 1 (MHA), odd page count
     (2, 260, 9, 1, [260, 259], 8, 1),              # G = 8
 ])
-def test_select_band_rule_and_scores(dd, B, P, k, forced, n_pages, G, Tq):
-    n_exact, n_all, _, _ = _select_case(dd, B, P, k, forced, n_pages, seed=P + k, G=G, Tq=Tq)
+@pytest.mark.parametrize("select_mode", [0, 1], ids=["fused", "two_kernels"])
+def test_select_band_rule_and_scores(dd, B, P, k, forced, n_pages, G, Tq, select_mode):
+    n_exact, n_all, got, _ = _select_case(dd, B, P, k, forced, n_pages, seed=P + k, G=G, Tq=Tq, select_mode=select_mode)
     assert n_exact >= 1 or n_all == 0
+    if select_mode == 0:       # both kernels take the decision in the same arithmetic: same sets, bit for bit
+        _, _, got2, _ = _select_case(dd, B, P, k, forced, n_pages, seed=P + k, G=G, Tq=Tq, select_mode=1)
+        assert np.array_equal(got, got2)
 
 
 def test_select_well_separated_scores_are_bit_exact(dd):
     """Sharper landmarks spread the scores, so nearly every (request, head) must match the oracle exactly."""
-    n_exact, n_all, got, want = _select_case(dd, 4, 1000, 20, 2, [1000, 990, 512, 77], seed=5, scale=3.0)
-    assert n_exact >= n_all - 2
-    assert (got == want).mean() > 0.98
+    for mode in (0, 1):
+        n_exact, n_all, got, want = _select_case(dd, 4, 1000, 20, 2, [1000, 990, 512, 77], seed=5, scale=3.0,
+                                                 select_mode=mode)
+        assert n_exact >= n_all - 2
+        assert (got == want).mean() > 0.98
 
 
 def test_select_long_request_uses_the_global_key_path(dd):
     """More pages than fit in shared memory (config 5's regime, reduced): keys live in global scratch."""
-    n_exact, n_all, _, _ = _select_case(dd, 1, 20000, 300, 0, [19997], seed=11)
-    assert n_all == HKV
+    for mode in (0, 1):
+        n_exact, n_all, _, _ = _select_case(dd, 1, 20000, 300, 0, [19997], seed=11, select_mode=mode)
+        assert n_all == HKV
 
 
 def test_select_ties_go_to_the_lower_page(dd):
@@ -121,13 +128,14 @@ def test_select_ties_go_to_the_lower_page(dd):
     B, P, k, forced = 1, 200, 10, 2
     lm = torch.randn(1, HKV, 1, D).expand(1, HKV, P, D).contiguous().to(torch.bfloat16)
     q = torch.randn(1, 2, HQ, D).to(torch.bfloat16)
-    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, forced_recent_pages=forced)
-    idx = torch.empty((B, HKV, k), dtype=torch.int32, device="cuda")
-    c.select_topk(q.cuda(), 1, lm.cuda(), torch.tensor([P], dtype=torch.int32).cuda(), idx)
-    assert c.device_error() == (0, 0)
-    want = list(range(k - forced)) + [P - 2, P - 1]
-    assert all(idx.cpu().numpy()[0, h].tolist() == want for h in range(HKV))
-    c.close()
+    for mode in (0, 1):
+        c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, forced_recent_pages=forced, select_mode=mode)
+        idx = torch.empty((B, HKV, k), dtype=torch.int32, device="cuda")
+        c.select_topk(q.cuda(), 1, lm.cuda(), torch.tensor([P], dtype=torch.int32).cuda(), idx)
+        assert c.device_error() == (0, 0)
+        want = list(range(k - forced)) + [P - 2, P - 1]
+        assert all(idx.cpu().numpy()[0, h].tolist() == want for h in range(HKV))
+        c.close()
 
 
 @pytest.mark.parametrize("mode", ["loads", "bulk"])
