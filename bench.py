@@ -25,6 +25,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# per-launch traffic from the committed ncu captures (config 2 layer: 64 MiB gathered, 32 MiB of landmarks)
+NCU_TRAFFIC = {"gather_dram": 38.7e3 + 9.36e6, "gather_sysmem": 2097152 * 32, "attn_dram": 67.33e6 + 0.95e6,
+               "select_dram": 33.68e6}
+
 METRIC = "decode_tokens_per_s"
 UNIT = "tok/s"
 
@@ -105,11 +109,12 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # CPU oracle legs
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(w, n_layers_cap=32, min_seconds=10.0):
-    """Times the oracle, as it stands, on whole layers of the workload (all requests, one step):
-    selection from the speculated token, page gather, attention of both tokens. Returns tok/s scaled to
-    a full step of w.n_layers layers."""
-    import numpy as np
+def oracle_sample(w, n_layers_cap=4, min_seconds=10.0, max_steps_per_layer=12):
+    """Times the oracle, as it stands, on whole layers of the workload (all requests): selection from the
+    speculated token, page gather, attention of both tokens. A few layers' slabs are drawn; each is run
+    for several steps of fresh queries until about `min_seconds` of oracle work has been timed. Returns
+    tok/s scaled to full steps of w.n_layers layers."""
+    import torch
     from oracle import dd_oracle as orc
     from paper_2607_26475_b200 import workloads as wl
     try:
@@ -119,33 +124,36 @@ def oracle_sample(w, n_layers_cap=32, min_seconds=10.0):
         threads = 1
     ctx_len = wl.ctx_lens(w).numpy()
     npg = (ctx_len + w.page_tokens - 1) // w.page_tokens
-    layers, t_total = 0, 0.0
+    n_units, t_total, layers = 0, 0.0, 0
     split = {"select": 0.0, "gather": 0.0, "attn": 0.0}
     while layers < n_layers_cap and (layers == 0 or t_total < min_seconds):
         l = layers
-        import torch
-        kv = torch.stack([wl.kv_slab(w, l, b) for b in range(w.batch)])
-        kv32 = kv.float().numpy()
+        kv32 = torch.stack([wl.kv_slab(w, l, b) for b in range(w.batch)]).float().numpy()
         lm = orc.build_landmarks(kv32[:, :, :, 0], ctx_len)             # set-up, not timed
-        q = wl.queries(w, 0, l).float().numpy()
-        t0 = time.perf_counter()
-        idx, _ = orc.select_topk(q[:, 1], lm, npg, w.k_pages, w.forced_recent_pages)
-        t1 = time.perf_counter()
-        slot = orc.gather_kv(kv32, idx)
-        t2 = time.perf_counter()
-        orc.sparse_decode_attn(q, slot, idx, ctx_len, w.page_tokens)
-        t3 = time.perf_counter()
-        split["select"] += t1 - t0
-        split["gather"] += t2 - t1
-        split["attn"] += t3 - t2
-        t_total += t3 - t0
+        for step in range(max_steps_per_layer):
+            q = wl.queries(w, step, l).float().numpy()
+            t0 = time.perf_counter()
+            idx, _ = orc.select_topk(q[:, 1], lm, npg, w.k_pages, w.forced_recent_pages)
+            t1 = time.perf_counter()
+            slot = orc.gather_kv(kv32, idx)
+            t2 = time.perf_counter()
+            orc.sparse_decode_attn(q, slot, idx, ctx_len, w.page_tokens)
+            t3 = time.perf_counter()
+            split["select"] += t1 - t0
+            split["gather"] += t2 - t1
+            split["attn"] += t3 - t2
+            t_total += t3 - t0
+            n_units += 1
+            if t_total >= min_seconds:
+                break
         layers += 1
-        del kv, kv32, slot
-    per_layer = t_total / layers
+        del kv32, lm
+    per_layer = t_total / n_units
     value = w.batch / (per_layer * w.n_layers)
     return {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{layers} layer(s) x all {w.batch} requests x 1 step of {w.name}, scaled to {w.n_layers} layers",
-            "us_per_layer": {k: v / layers * 1e6 for k, v in split.items()}, "seconds": t_total}
+            "sample": f"{n_units} layer-steps (all {w.batch} requests; {layers} layer(s) x up to {max_steps_per_layer} "
+                      f"steps) of {w.name}, scaled to {w.n_layers} layers per step",
+            "us_per_layer": {k: v / n_units * 1e6 for k, v in split.items()}, "seconds": t_total}
 
 
 def run_reference(args):
@@ -155,11 +163,11 @@ def run_reference(args):
     from paper_2607_26475_b200 import workloads as wl
     w = wl.CONFIGS[args.config]
     for _ in range(min(args.warmup, 1)):
-        oracle_sample(w, n_layers_cap=1, min_seconds=0.0)
+        oracle_sample(w, n_layers_cap=1, min_seconds=0.0, max_steps_per_layer=1)
     vals, info = [], None
     t0 = time.time()
     for _ in range(args.steps):
-        info = oracle_sample(w, n_layers_cap=1, min_seconds=0.0)
+        info = oracle_sample(w, n_layers_cap=1, min_seconds=0.0, max_steps_per_layer=1)
         vals.append(info["value"])
         if time.time() - t0 > 150:
             break
@@ -187,6 +195,7 @@ def main():
     import torch.distributed as dist
     from paper_2607_26475_b200 import binding as dd
     from paper_2607_26475_b200 import workloads as wl
+    from paper_2607_26475_b200 import replicas
     from paper_2607_26475_b200.store import HostStore, available_host_bytes
 
     rank = int(os.environ.get("RANK", "0"))
@@ -207,7 +216,7 @@ def main():
     ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                      forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
                      gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy)
-    budget = int(available_host_bytes() * 0.6 / max(1, world))
+    budget = replicas.host_budget_per_rank(available_host_bytes(), world)
     store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, host_budget_bytes=budget,
                       log=log if rank == 0 else None)
     store.bind(ctx)
@@ -277,12 +286,9 @@ def main():
     code, detail = ctx.device_error()
     if code != 0:
         raise RuntimeError(f"device error {code} (detail {detail}) during the timed run")
-    t_ms = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_total = float(t_ms.item())
+    ms_total, tokens = replicas.aggregate(ms_total, B * K, device="cuda")
     ms_per_step = ms_total / K
-    value = world * B * K / (ms_total * 1e-3)
+    value = tokens / (ms_total * 1e-3)
     n_gathers = K * L
     gather_bytes = w.gathered_bytes_per_layer
     gather_ms_live = copy_ms / n_gathers
@@ -314,10 +320,7 @@ def main():
         compute.wait_event(tail)
         e1.record(compute)
     barrier()
-    t_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    e2e_value = world * B * K / (float(t_ms.item()) * 1e-3)
+    e2e_value = replicas.throughput(e0.elapsed_time(e1), B * K, device="cuda")
     q_bytes = q_step.numel() * 2
     o_bytes = outs.numel() * 2
 
@@ -345,12 +348,16 @@ def main():
     if rank == 0:
         us_layer = ms_per_step / L * 1e3
         link_time_us = gather_bytes / (link_peak * 1e9) * 1e6
-        hbm_bytes = (B * w.n_kv_heads * w.n_pages * 256 * 1.125) + 2 * gather_bytes
+        hbm_bytes = (B * w.n_kv_heads * w.n_pages * 256) + 2 * gather_bytes
         hbm_time_us = hbm_bytes / (hbm_peak * 1e9) * 1e6
         line["roofline"] = {
             "kernel": "dd_gather_loads_kernel" if args.gather_mode == "loads" else "dd_gather_bulk_kernel",
             "bound": "host_link", "achieved": gather_bytes / (gather_ms_live * 1e-3) / 1e9, "peak": link_peak,
-            "unit": "GB/s", "frac": gather_bytes / (gather_ms_live * 1e-3) / 1e9 / link_peak, "traffic": None,
+            "unit": "GB/s", "frac": gather_bytes / (gather_ms_live * 1e-3) / 1e9 / link_peak,
+            "traffic": NCU_TRAFFIC["gather_dram"] * gather_bytes / (64 << 20),
+            "link_traffic": NCU_TRAFFIC["gather_sysmem"] * gather_bytes / (64 << 20),
+            "traffic_source": "ncu capture of a 64 MiB launch (profiles/dd_gather_kernels_config2.md), scaled by gathered "
+                              "bytes: `traffic` = DRAM read+write (the slot stays in L2), `link_traffic` = sysmem sectors x 32 B",
             "peak_source": "pinned cudaMemcpyAsync host->device, 256 MiB, best of 6, measured in this run",
             "how": "gathered bytes per launch / (copy-stream span of the timed region / launches)",
         }
@@ -444,17 +451,19 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     torch.cuda.synchronize()
     compute_only = e0.elapsed_time(e1) * 1e3 / (n_rep * L)
     lm_bytes = B * w.n_kv_heads * w.n_pages * 256
-    sel_bytes = lm_bytes * 1.125          # landmarks once + fp32 logits written and read (4 heads x 4 B per 256 B row, twice)
+    sel_bytes = float(lm_bytes)           # landmarks once; the fused kernel keeps the logits in shared memory
     gb = w.gathered_bytes_per_layer
     return {
         "select_us": sel_us, "gather_us": gat_us, "attn_us_l2_warm": att_warm, "attn_us_l2_flushed": att_cold,
         "compute_only_us_per_layer": compute_only, "reps": reps,
         "roofline_kernels": {
-            "select(dd_score_kernel+dd_topk_kernel)": {"bound": "hbm", "achieved": sel_bytes / (sel_us * 1e-6) / 1e9,
-                                                       "peak": hbm_peak, "unit": "GB/s",
-                                                       "frac": sel_bytes / (sel_us * 1e-6) / 1e9 / hbm_peak},
+            "dd_select_fused_kernel": {"bound": "hbm", "achieved": sel_bytes / (sel_us * 1e-6) / 1e9,
+                                       "peak": hbm_peak, "unit": "GB/s",
+                                       "frac": sel_bytes / (sel_us * 1e-6) / 1e9 / hbm_peak,
+                                       "traffic": NCU_TRAFFIC["select_dram"] * lm_bytes / (32 << 20)},
             "dd_attn_kernel(l2 flushed)": {"bound": "hbm", "achieved": gb / (att_cold * 1e-6) / 1e9, "peak": hbm_peak,
-                                           "unit": "GB/s", "frac": gb / (att_cold * 1e-6) / 1e9 / hbm_peak},
+                                           "unit": "GB/s", "frac": gb / (att_cold * 1e-6) / 1e9 / hbm_peak,
+                                           "traffic": NCU_TRAFFIC["attn_dram"] * gb / (64 << 20)},
             "gather(alone)": {"bound": "host_link", "achieved": gb / (gat_us * 1e-6) / 1e9, "peak": link_peak,
                               "unit": "GB/s", "frac": gb / (gat_us * 1e-6) / 1e9 / link_peak},
         },
