@@ -46,6 +46,8 @@ __all__ = [
     "gather_kv",
     "sparse_decode_attn",
     "decode_chain",
+    "correct_misses",
+    "decode_chain_corrected",
 ]
 
 
@@ -238,3 +240,57 @@ def decode_chain(q_init: np.ndarray, q_steps: np.ndarray, lm_layers, kv_layers, 
             outs[t, l], _ = sparse_decode_attn(q_steps[t, l], slot, idxs[t, l], ctx_len, page_tokens)
             idxs[t + 1, l], _ = select_topk(q_steps[t, l][:, 1], lm_layers[l], n_pages, k, forced_recent)
     return outs, idxs
+
+
+def correct_misses(pred_idx: np.ndarray, true_idx: np.ndarray):
+    """Repair of a predicted set once the true index is known (Sec. 5.3 "Prioritized missing KV transfer":
+    the pages the prediction missed are fetched before attention so that the result is the one computed
+    with the true retrieval index; Sec. 5.4: the assembly step merges them into the layer's buffer).
+
+    pred_idx, true_idx [B, Hkv, k] ascending. The pages of the true set the prediction lacks
+    (missing = true \ predicted, ascending) take the buffer positions of the pages the true set does not
+    want (victims = predicted \ true, in ascending position). Returns
+      merged  [B, Hkv, k]  page held by every buffer position after the repair (as a set = the true set),
+      fixes   list over (b, g) of (positions, pages) arrays,
+      n_miss  [B, Hkv]."""
+    B, Hkv, k = pred_idx.shape
+    merged = np.array(pred_idx, dtype=np.int32, copy=True)
+    fixes = []
+    n_miss = np.zeros((B, Hkv), dtype=np.int32)
+    for b in range(B):
+        for g in range(Hkv):
+            pred = [int(x) for x in pred_idx[b, g]]
+            true = [int(x) for x in true_idx[b, g]]
+            pred_set, true_set = set(pred), set(true)
+            missing = [p for p in true if p not in pred_set]
+            victims = [j for j, p in enumerate(pred) if p not in true_set]
+            assert len(missing) == len(victims)
+            for j, p in zip(victims, missing):
+                merged[b, g, j] = p
+            fixes.append((np.array(victims, dtype=np.int32), np.array(missing, dtype=np.int32)))
+            n_miss[b, g] = len(missing)
+    return merged, fixes, n_miss
+
+
+def decode_chain_corrected(q_init: np.ndarray, q_steps: np.ndarray, lm_layers, kv_layers, n_pages: np.ndarray,
+                           ctx_len: np.ndarray, k: int, page_tokens: int, forced_recent: int = 0):
+    """The chain with miss correction: the set prefetched for step t is predicted from the speculated token
+    of step t-1 (or q_init), the true set comes from the current token of step t, and attention runs over
+    the repaired buffer, i.e. over the true set (Sec. 4.2: prediction does not change the attention result).
+    Returns (outs [S, L, B, 2, Hq, d], pred [S+1, L, B, Hkv, k], true [S, L, B, Hkv, k], n_miss [S, L, B, Hkv])."""
+    S, L, B = q_steps.shape[0], q_steps.shape[1], q_steps.shape[2]
+    Hkv = lm_layers[0].shape[1]
+    pred = np.empty((S + 1, L, B, Hkv, k), dtype=np.int32)
+    true = np.empty((S, L, B, Hkv, k), dtype=np.int32)
+    n_miss = np.empty((S, L, B, Hkv), dtype=np.int32)
+    outs = np.empty(q_steps.shape, dtype=np.float64)
+    for l in range(L):
+        pred[0, l], _ = select_topk(q_init[l], lm_layers[l], n_pages, k, forced_recent)
+    for t in range(S):
+        for l in range(L):
+            true[t, l], _ = select_topk(q_steps[t, l][:, 0], lm_layers[l], n_pages, k, forced_recent)
+            merged, _, n_miss[t, l] = correct_misses(pred[t, l], true[t, l])
+            slot = gather_kv(kv_layers[l], merged)
+            outs[t, l], _ = sparse_decode_attn(q_steps[t, l], slot, merged, ctx_len, page_tokens)
+            pred[t + 1, l], _ = select_topk(q_steps[t, l][:, 1], lm_layers[l], n_pages, k, forced_recent)
+    return outs, pred, true, n_miss

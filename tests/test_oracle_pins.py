@@ -319,3 +319,53 @@ def test_chain_uses_the_speculated_token_of_the_previous_step():
     q2[:, :, :, 0] += 5.0
     _, idxs2 = orc.decode_chain(q_init, q2, lm, kv, npg, ctx, k, T)
     assert np.array_equal(idxs, idxs2)
+
+
+# ----------------------------------------------------------------------------- miss correction
+def test_correction_hand_example_and_set_identities():
+    """Predicted {1,4,6,9}, true {2,4,9,11}: pages 2 and 11 are missing, the victims are positions 0 and 2
+    (pages 1 and 6). After the repair the buffer holds [2, 4, 11, 9]."""
+    pred = np.array([[[1, 4, 6, 9]]], dtype=np.int32)
+    true = np.array([[[2, 4, 9, 11]]], dtype=np.int32)
+    merged, fixes, n_miss = orc.correct_misses(pred, true)
+    assert merged.tolist() == [[[2, 4, 11, 9]]]
+    assert fixes[0][0].tolist() == [0, 2] and fixes[0][1].tolist() == [2, 11]
+    assert n_miss.tolist() == [[1 * 2]]
+    rng = np.random.default_rng(20)
+    for _ in range(30):
+        P, k = 60, 17
+        a = np.sort(rng.choice(P, k, replace=False)).astype(np.int32)[None, None]
+        b = np.sort(rng.choice(P, k, replace=False)).astype(np.int32)[None, None]
+        merged, fixes, n_miss = orc.correct_misses(a, b)
+        assert set(merged[0, 0].tolist()) == set(b[0, 0].tolist())            # the buffer holds the true set
+        keep = [j for j in range(k) if a[0, 0, j] in set(b[0, 0].tolist())]
+        assert all(merged[0, 0, j] == a[0, 0, j] for j in keep)                # common pages do not move
+        assert n_miss[0, 0] == len(set(b[0, 0].tolist()) - set(a[0, 0].tolist()))
+        assert np.all(np.diff(fixes[0][0]) > 0) and np.all(np.diff(fixes[0][1]) > 0)
+    same, fixes, n_miss = orc.correct_misses(pred, pred)
+    assert np.array_equal(same, pred) and n_miss.sum() == 0 and fixes[0][0].size == 0
+
+
+def test_corrected_chain_equals_attention_over_the_true_sets():
+    """With correction the prediction must not change the result: every output equals attention over the
+    set selected from the current token, whatever was predicted."""
+    rng = np.random.default_rng(21)
+    S, L, B, Hq, Hkv, P, T, d, k = 2, 2, 2, 4, 2, 12, 2, 8, 4
+    ctx = np.array([P * T, P * T - 1])
+    npg = np.array([P, P])
+    kv = [orc.round_to_bf16(rng.standard_normal((B, Hkv, P, 2, T, d)).astype(np.float32)) for _ in range(L)]
+    lm = [orc.build_landmarks(kv[l][:, :, :, 0], ctx) for l in range(L)]
+    q_init = rng.standard_normal((L, B, Hq, d))
+    q_steps = rng.standard_normal((S, L, B, 2, Hq, d))
+    outs, pred, true, n_miss = orc.decode_chain_corrected(q_init, q_steps, lm, kv, npg, ctx, k, T)
+    assert n_miss.sum() > 0                                    # independent tokens: the prediction does miss
+    for t in range(S):
+        for l in range(L):
+            want_true, _ = orc.select_topk(q_steps[t, l][:, 0], lm[l], npg, k)      # token 0 = current
+            assert np.array_equal(true[t, l], want_true)
+            o, _ = orc.sparse_decode_attn(q_steps[t, l], orc.gather_kv(kv[l], want_true), want_true, ctx, T)
+            np.testing.assert_allclose(outs[t, l], o, rtol=1e-12, atol=1e-14)
+    # another priming query changes the first prediction but not a single output
+    outs2, pred2, _, _ = orc.decode_chain_corrected(q_init + 3.0, q_steps, lm, kv, npg, ctx, k, T)
+    assert not np.array_equal(pred[0], pred2[0])
+    np.testing.assert_allclose(outs, outs2, rtol=1e-12, atol=1e-14)
