@@ -51,6 +51,8 @@ def parse_args():
     ap.add_argument("--attn-splits", type=int, default=0)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling of small cases only)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of small cases only)")
+    ap.add_argument("--correct-misses", action="store_true",
+                    help="repair prediction misses on an urgent stream before attention (not the headline path)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
     return ap.parse_args()
@@ -212,10 +214,12 @@ def main():
 
     compute = torch.cuda.Stream()
     copy = torch.cuda.Stream(priority=0)
+    urgent = torch.cuda.Stream(priority=-1) if args.correct_misses else None
     gm = dd.DD_GATHER_BULK if args.gather_mode == "bulk" else dd.DD_GATHER_LOADS
     ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                      forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
-                     gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy)
+                     gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy,
+                     miss_correction=args.correct_misses, urgent_stream=urgent)
     budget = replicas.host_budget_per_rank(available_host_bytes(), world)
     store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, host_budget_bytes=budget,
                       log=log if rank == 0 else None)
@@ -286,6 +290,7 @@ def main():
     code, detail = ctx.device_error()
     if code != 0:
         raise RuntimeError(f"device error {code} (detail {detail}) during the timed run")
+    miss = ctx.miss_stats(reset=True) if args.correct_misses else None
     ms_total, tokens = replicas.aggregate(ms_total, B * K, device="cuda")
     ms_per_step = ms_total / K
     value = tokens / (ms_total * 1e-3)
@@ -341,10 +346,16 @@ def main():
                 "d2h_bytes_per_step": o_bytes,
                 "note": "queries copied from pinned host memory and outputs read back every step, host waits for "
                         "each step; the KV gather from the host store is part of the path in both numbers"},
-        "gpu_launches": K * L * 4,
+        "gpu_launches": K * L * (7 if args.correct_misses else 3),
         "clocks": clocks,
     }
 
+    if miss is not None:
+        line["miss_correction"] = {"missing_pages": miss[0], "selected_pages": miss[1],
+                                   "miss_rate": miss[0] / max(1, miss[1]),
+                                   "extra_link_bytes_per_layer": miss[0] * w.page_bytes / max(1, (W + K) * L),
+                                   "note": "attention runs over the set selected from the current token; the pages the "
+                                           "prediction missed cross the link on the urgent stream (counts include warm-up)"}
     if rank == 0:
         us_layer = ms_per_step / L * 1e3
         link_time_us = gather_bytes / (link_peak * 1e9) * 1e6
@@ -365,7 +376,7 @@ def main():
                               "frac_of_roofline": max(link_time_us, hbm_time_us) / us_layer,
                               "link_us": link_time_us, "hbm_us": hbm_time_us, "hbm_peak_gbs": hbm_peak,
                               "hbm_peak_source": peak_src}
-        if not args.no_stages:
+        if not args.no_stages and not args.correct_misses:
             line["stages"] = stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, args, K, W)
             st = line["stages"]
             t_c = st["compute_only_us_per_layer"]

@@ -74,6 +74,8 @@ typedef struct dd_config {
   void* copy_stream;         /* cudaStream_t used by the pipelined calls for the gather */
   void* ring_mem;            /* optional caller-owned ring of dd_ring_bytes(); NULL = library allocates */
   size_t ring_bytes;         /* size of ring_mem when supplied */
+  int miss_correction;       /* 1: dd_decode_layer_step repairs prediction misses before attention (needs urgent_stream) */
+  void* urgent_stream;       /* cudaStream_t, ideally of higher priority than copy_stream; used for the missing pages */
 } dd_config;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -184,8 +186,31 @@ int dd_prime(dd_ctx* ctx, const void* q_init);
  *   out  dev bf16 [B][Tq][Hq][d], written */
 int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out);
 
-/* Device address of the index set [B][Hkv][k] that attention uses at (step parity, layer). No copy. */
+/* Device address of the predicted index set [B][Hkv][k] prefetched for (step parity, layer). No copy. */
 int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx);
+
+/* ---- miss correction (Sec. 5.3 "Prioritized missing KV transfer") --------------------------------- */
+
+/* With dd_config.miss_correction = 1, dd_decode_layer_step first selects the TRUE index of the layer from
+ * the current token (token 0 of q), compares it with the predicted set that was prefetched into the slot,
+ * fetches the missing pages (true minus predicted) on urgent_stream into the buffer positions of the pages
+ * the true set does not contain, and runs attention over the repaired slot — i.e. over the true set, so the
+ * prediction no longer influences the result (Sec. 4.2). The selection for the next step runs on the
+ * compute stream while the urgent transfer is in flight. The two calls below are that repair in pieces.
+ *
+ * dd_diff_indices: pred_idx, true_idx dev int32 [B][Hkv][k], both ascending. Writes merged_idx
+ * (dev int32 [B][Hkv][k]): position j keeps pred_idx[j] when that page is in the true set, else takes the
+ * next missing page in ascending order; as a set, merged_idx equals true_idx. Also fills the context's fix
+ * list of ring slot `slot` and adds to the miss statistics. Asynchronous on `stream`. */
+int dd_diff_indices(dd_ctx* ctx, const int* pred_idx, const int* true_idx, int slot, int* merged_idx, void* stream);
+/* dd_fetch_missing_from_host: copies the pages on the fix list of `slot` (written by the last
+ * dd_diff_indices for that slot, which must precede this call in stream order) from host_kv_layer
+ * (pinned or dev, bf16 [B][Hkv][P][2][T][d]) into their positions of the slot. Asynchronous on `stream`. */
+int dd_fetch_missing_from_host(dd_ctx* ctx, const void* host_kv_layer, int slot, void* stream);
+/* Device address of the repaired page list [B][Hkv][k] of ring slot `slot` (valid after a corrected layer step). */
+int dd_get_merged_indices(dd_ctx* ctx, int slot, const int** dev_idx);
+/* Synchronises, then reports how many pages were missing and how many were selected since the last reset. */
+int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset);
 
 /* ---- attention without any allocation ----------------------------------------------------------- */
 

@@ -248,8 +248,8 @@ def correct_misses(pred_idx: np.ndarray, true_idx: np.ndarray):
     with the true retrieval index; Sec. 5.4: the assembly step merges them into the layer's buffer).
 
     pred_idx, true_idx [B, Hkv, k] ascending. The pages of the true set the prediction lacks
-    (missing = true \ predicted, ascending) take the buffer positions of the pages the true set does not
-    want (victims = predicted \ true, in ascending position). Returns
+    (missing = true minus predicted, ascending) take the buffer positions of the pages the true set does not
+    want (victims = predicted minus true, in ascending position). Returns
       merged  [B, Hkv, k]  page held by every buffer position after the repair (as a set = the true set),
       fixes   list over (b, g) of (positions, pages) arrays,
       n_miss  [B, Hkv]."""

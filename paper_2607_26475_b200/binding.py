@@ -33,6 +33,7 @@ EXPORTS = [
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
+    "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
 ]
 
 
@@ -45,6 +46,7 @@ class DDConfig(C.Structure):
         ("gather_mode", C.c_int), ("gather_ctas", C.c_int), ("select_mode", C.c_int), ("attn_splits", C.c_int),
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
+        ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
     ]
 
 
@@ -80,6 +82,10 @@ def _load() -> C.CDLL:
     lib.dd_prime.argtypes = [vp, vp]
     lib.dd_decode_layer_step.argtypes = [vp, ip, ip, vp, vp]
     lib.dd_get_indices.argtypes = [vp, ip, ip, C.POINTER(vp)]
+    lib.dd_diff_indices.argtypes = [vp, vp, vp, ip, vp, vp]
+    lib.dd_fetch_missing_from_host.argtypes = [vp, vp, ip, vp]
+    lib.dd_get_merged_indices.argtypes = [vp, ip, C.POINTER(vp)]
+    lib.dd_miss_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong), ip]
     lib.dd_static_scratch_capacity.argtypes = []
     lib.dd_static_scratch_capacity.restype = C.c_size_t
     lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7
@@ -138,16 +144,22 @@ class Context:
 
     def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
-                 gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None):
+                 gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None,
+                 miss_correction=False, urgent_stream=None):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
         self.copy_stream = copy_stream if copy_stream is not None else torch.cuda.Stream()
         self._ring = ring
+        self.urgent_stream = urgent_stream
+        if miss_correction and urgent_stream is None:
+            self.urgent_stream = torch.cuda.Stream(priority=-1)
         self.cfg = DDConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, page_tokens, max_pages, k_pages,
                             forced_recent_pages, n_q_tokens, ring_depth, gather_mode, gather_ctas, select_mode, attn_splits,
                             self.compute_stream.cuda_stream, self.copy_stream.cuda_stream,
-                            _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0)
+                            _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0,
+                            1 if miss_correction else 0,
+                            self.urgent_stream.cuda_stream if self.urgent_stream is not None else None)
         self._h = C.c_void_p()
         self._keep = []
         rc = lib.dd_create(C.byref(self.cfg), C.byref(self._h))
@@ -230,6 +242,26 @@ class Context:
 
     def decode_layer_step(self, step, layer, q, out):
         self._check(lib.dd_decode_layer_step(self._h, step, layer, _ptr(q), _ptr(out)))
+
+    def diff_indices(self, pred_idx, true_idx, slot, merged_idx, stream=None):
+        self._check(lib.dd_diff_indices(self._h, _ptr(pred_idx), _ptr(true_idx), slot, _ptr(merged_idx), _stream(stream)))
+
+    def fetch_missing_from_host(self, host_kv_layer, slot, stream=None):
+        self._check(lib.dd_fetch_missing_from_host(self._h, _ptr(host_kv_layer), slot, _stream(stream)))
+
+    def get_merged_indices(self, slot) -> torch.Tensor:
+        """A copy of the repaired page list [B, Hkv, k] int32 of ring slot `slot` (synchronises)."""
+        p = C.c_void_p()
+        self._check(lib.dd_get_merged_indices(self._h, slot, C.byref(p)))
+        c = self.cfg
+        torch.cuda.synchronize()
+        return _view(p.value, (c.batch, c.n_kv_heads, c.k_pages), "i4").clone()
+
+    def miss_stats(self, reset=False):
+        """(missing pages, selected pages) accumulated by the corrected layer steps (synchronises)."""
+        a, b = C.c_ulonglong(), C.c_ulonglong()
+        self._check(lib.dd_miss_stats(self._h, C.byref(a), C.byref(b), 1 if reset else 0))
+        return a.value, b.value
 
     def get_indices(self, step_parity, layer) -> torch.Tensor:
         """A copy of the index set [B, Hkv, k] int32 used at (step parity, layer) (synchronises)."""

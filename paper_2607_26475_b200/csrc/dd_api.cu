@@ -58,6 +58,7 @@ static const char* dd_check_config(const dd_config* c) {
   if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK) return "unknown gather_mode";
   if (c->select_mode != DD_SELECT_AUTO && c->select_mode != DD_SELECT_TWO_KERNELS) return "unknown select_mode";
   if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
+  if (c->miss_correction != 0 && c->miss_correction != 1) return "miss_correction must be 0 or 1";
   if (c->attn_splits > 512) return "attn_splits must be <= 512";
   if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";
   if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
@@ -94,8 +95,12 @@ static int dd_resolve_splits(const dd_config* c, int sm_count, int* cluster_out)
 }
 
 struct dd_sizes {
-  size_t score_s, score_part, topk_keys, part_o, part_ml, ticket, idx_tab, err;
-  size_t total() const { return score_s + score_part + topk_keys + part_o + part_ml + ticket + idx_tab + err; }
+  size_t score_s, score_part, topk_keys, part_o, part_ml, ticket, idx_tab, err, idx_true, idx_merged, fix_stage, fix_list,
+      fix_count, stats;
+  size_t total() const {
+    return score_s + score_part + topk_keys + part_o + part_ml + ticket + idx_tab + err + idx_true + idx_merged +
+           fix_stage + fix_list + fix_count + stats;
+  }
 };
 
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -112,6 +117,13 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
   z.ticket = up256(B * Hkv * 4);
   z.idx_tab = up256((size_t)2 * c->n_layers * B * Hkv * c->k_pages * 4);
   z.err = 256;
+  const size_t sel = B * Hkv * (size_t)c->k_pages, D = c->ring_depth;
+  z.idx_true = up256(sel * 4);
+  z.idx_merged = up256(D * sel * 4);
+  z.fix_stage = up256(D * sel * 8);
+  z.fix_list = up256(D * sel * 16);
+  z.fix_count = 256;
+  z.stats = 256;
   return z;
 }
 
@@ -141,6 +153,8 @@ static void dd_free_all(dd_ctx* ctx) {
   for (int i = 0; i < DD_MAX_RING; ++i) {
     if (ctx->ready[i]) cudaEventDestroy(ctx->ready[i]);
     if (ctx->released[i]) cudaEventDestroy(ctx->released[i]);
+    if (ctx->fix_ready[i]) cudaEventDestroy(ctx->fix_ready[i]);
+    if (ctx->urgent_done[i]) cudaEventDestroy(ctx->urgent_done[i]);
   }
   if (ctx->sel_done) {
     for (int l = 0; l < ctx->cfg.n_layers; ++l)
@@ -156,6 +170,8 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   if (!out) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: out is NULL");
   *out = nullptr;
   if (const char* why = dd_check_config(cfg)) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: %s", why);
+  if (cfg->miss_correction && !cfg->urgent_stream)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: miss_correction needs an urgent_stream of its own");
   dd_ctx* ctx = new (std::nothrow) dd_ctx();
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: out of host memory");
   memset(ctx, 0, sizeof(*ctx));
@@ -193,10 +209,18 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   ctx->attn_part_ml = (float2*)base;                 base += z.part_ml;
   ctx->attn_ticket = (unsigned int*)base;            base += z.ticket;
   ctx->idx_tab = (int*)base;                         base += z.idx_tab;
-  ctx->err_word = (int*)base;
+  ctx->err_word = (int*)base;                        base += z.err;
+  ctx->idx_true = (int*)base;                        base += z.idx_true;
+  ctx->idx_merged = (int*)base;                      base += z.idx_merged;
+  ctx->fix_stage = (int2*)base;                      base += z.fix_stage;
+  ctx->fix_list = (int4*)base;                       base += z.fix_list;
+  ctx->fix_count = (unsigned int*)base;              base += z.fix_count;
+  ctx->miss_stats = (unsigned long long*)base;
   DD_CREATE_TRY(cudaMemset(ctx->attn_ticket, 0, z.ticket));
   DD_CREATE_TRY(cudaMemset(ctx->idx_tab, 0, z.idx_tab));
   DD_CREATE_TRY(cudaMemset(ctx->err_word, 0, z.err));
+  DD_CREATE_TRY(cudaMemset(ctx->fix_count, 0, z.fix_count));
+  DD_CREATE_TRY(cudaMemset(ctx->miss_stats, 0, z.stats));
   if (cfg->ring_mem) {
     if (cfg->ring_bytes < dd_ring_bytes(cfg)) {
       int rc = dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_create: ring_mem holds %zu bytes, %zu needed", cfg->ring_bytes,
@@ -217,6 +241,8 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   for (int i = 0; i < cfg->ring_depth; ++i) {
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->ready[i], cudaEventDisableTiming));
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->released[i], cudaEventDisableTiming));
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->fix_ready[i], cudaEventDisableTiming));
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->urgent_done[i], cudaEventDisableTiming));
   }
   ctx->sel_done = new cudaEvent_t[cfg->n_layers]();
   for (int l = 0; l < cfg->n_layers; ++l)
@@ -239,8 +265,9 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
 extern "C" int dd_sync(dd_ctx* ctx, double timeout_s) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sync: ctx is NULL");
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(timeout_s);
-  cudaStream_t streams[2] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream};
-  for (int i = 0; i < 2; ++i) {
+  cudaStream_t streams[3] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream,
+                             (cudaStream_t)ctx->cfg.urgent_stream};
+  for (int i = 0; i < (ctx->cfg.miss_correction ? 3 : 2); ++i) {
     for (;;) {
       cudaError_t e = cudaStreamQuery(streams[i]);
       if (e == cudaSuccess) break;
@@ -457,14 +484,37 @@ extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void
   cudaStream_t cs = (cudaStream_t)c.compute_stream;
   const int slot = (int)(n % c.ring_depth);
 
-  DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));                    // transfer complete
-  DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, dd_idx_of(ctx, step, layer), ctx->ctx_len,
-                        out, nullptr, cs));
+  const int spec_token = c.n_q_tokens - 1;
+  const int* attn_idx = dd_idx_of(ctx, step, layer);
+  if (c.miss_correction) {
+    // true index from the current token, repair list, missing pages on the urgent stream; the selection for
+    // the next step runs on the compute stream while that transfer is in flight
+    cudaStream_t us = (cudaStream_t)c.urgent_stream;
+    int* merged = ctx->idx_merged + (size_t)slot * c.batch * c.n_kv_heads * c.k_pages;
+    DD_TRY(dd_launch_select(ctx, q, 0, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages, ctx->idx_true, nullptr, cs));
+    DD_TRY(dd_launch_diff(ctx, attn_idx, ctx->idx_true, slot, merged, cs));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->fix_ready[slot], cs));
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->fix_ready[slot], 0));
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->ready[slot], 0));                  // the prefetch wrote the slot first
+    DD_TRY(dd_launch_gather_fix(ctx, ctx->host_kv[layer], slot, us));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->urgent_done[slot], us));
+    DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
+                            dd_idx_of(ctx, step + 1, layer), nullptr, cs));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->urgent_done[slot], 0));            // all transfers of the layer complete
+    attn_idx = merged;
+  } else {
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));                  // transfer complete
+  }
+  DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, attn_idx, ctx->ctx_len, out, nullptr, cs));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
   ctx->released_recorded[slot] = true;
-  DD_TRY(dd_launch_select(ctx, q, c.n_q_tokens - 1, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
-                          dd_idx_of(ctx, step + 1, layer), nullptr, cs));
-  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+  if (!c.miss_correction) {
+    DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
+                            dd_idx_of(ctx, step + 1, layer), nullptr, cs));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+  }
   // the slot just released takes the gather `ahead` layers further on (index set known: it was
   // selected one step earlier, or just now when the ring is deeper than the model)
   const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
@@ -477,5 +527,45 @@ extern "C" int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int
   if (!ctx || !dev_idx) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_get_indices: NULL argument");
   if (layer < 0 || layer >= ctx->cfg.n_layers) return dd_fail(ctx, DD_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
   *dev_idx = dd_idx_of(ctx, step_parity, layer);
+  return DD_OK;
+}
+
+extern "C" int dd_diff_indices(dd_ctx* ctx, const int* pred_idx, const int* true_idx, int slot, int* merged_idx,
+                               void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_diff_indices: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  DD_TRY(dd_check_dev(ctx, pred_idx, "pred_idx", 4));
+  DD_TRY(dd_check_dev(ctx, true_idx, "true_idx", 4));
+  DD_TRY(dd_check_dev(ctx, merged_idx, "merged_idx", 4));
+  return dd_launch_diff(ctx, pred_idx, true_idx, slot, merged_idx, (cudaStream_t)stream);
+}
+
+extern "C" int dd_fetch_missing_from_host(dd_ctx* ctx, const void* host_kv_layer, int slot, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_fetch_missing_from_host: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  const void* kv_dev = nullptr;
+  DD_TRY(dd_check_store(ctx, host_kv_layer, "host_kv_layer", &kv_dev));
+  return dd_launch_gather_fix(ctx, kv_dev, slot, (cudaStream_t)stream);
+}
+
+extern "C" int dd_get_merged_indices(dd_ctx* ctx, int slot, const int** dev_idx) {
+  if (!ctx || !dev_idx) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_get_merged_indices: NULL argument");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  *dev_idx = ctx->idx_merged + (size_t)slot * ctx->cfg.batch * ctx->cfg.n_kv_heads * ctx->cfg.k_pages;
+  return DD_OK;
+}
+
+extern "C" int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_miss_stats: ctx is NULL");
+  DD_TRY(dd_sync(ctx, 60.0));
+  DD_CUDA_TRY(ctx, cudaDeviceSynchronize());
+  unsigned long long w[2] = {0, 0};
+  DD_CUDA_TRY(ctx, cudaMemcpy(w, ctx->miss_stats, sizeof(w), cudaMemcpyDeviceToHost));
+  if (reset) DD_CUDA_TRY(ctx, cudaMemset(ctx->miss_stats, 0, sizeof(w)));
+  if (missing) *missing = w[0];
+  if (selected) *selected = w[1];
   return DD_OK;
 }

@@ -38,6 +38,13 @@ struct dd_ctx {
   unsigned int* attn_ticket;  // [B*Hkv] arrival counters, zero between launches
   int* idx_tab;          // [2][L][B][Hkv][k]
   int* err_word;         // [2]: code, detail
+  // miss correction
+  int* idx_true;         // [B][Hkv][k] true index of the layer being corrected
+  int* idx_merged;       // [D][B][Hkv][k] page held by every position of a slot after the repair
+  int2* fix_stage;       // [D][B][Hkv][k] per-unit (victim position, missing page) before pairing
+  int4* fix_list;        // [D][B*Hkv*k] compact (unit, position, page, 0)
+  unsigned int* fix_count;          // [D]
+  unsigned long long* miss_stats;   // [2]: missing pages, selected pages
   char* ring;
   bool own_ring;
   // events of the pipelined path
@@ -45,6 +52,8 @@ struct dd_ctx {
   cudaEvent_t released[DD_MAX_RING];
   bool released_recorded[DD_MAX_RING];
   cudaEvent_t* sel_done;  // [L]
+  cudaEvent_t fix_ready[DD_MAX_RING];    // fix list of the slot written (compute stream)
+  cudaEvent_t urgent_done[DD_MAX_RING];  // missing pages of the slot fetched (urgent stream)
   // bound tables
   const void** landmarks;  // [L]
   const void** host_kv;    // [L] device-visible addresses
@@ -69,6 +78,8 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
 int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int* n_pages, char* slot, cudaStream_t st);
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
                    float* out_lse, cudaStream_t st);
+int dd_launch_diff(dd_ctx* ctx, const int* pred, const int* truth, int slot, int* merged, cudaStream_t st);
+int dd_launch_gather_fix(dd_ctx* ctx, const void* kv_dev, int slot, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // device helpers
