@@ -53,6 +53,12 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of small cases only)")
     ap.add_argument("--correct-misses", action="store_true",
                     help="repair prediction misses on an urgent stream before attention (not the headline path)")
+    ap.add_argument("--urgent-fifo", action="store_true",
+                    help="with --correct-misses: queue the missing pages on the prefetch stream (single FIFO) instead "
+                         "of a high-priority stream of their own")
+    ap.add_argument("--spec-fidelity", type=float, default=None,
+                    help="override the generator's correlation between a step's speculated query and the next "
+                         "step's current query (lower = more prediction misses)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
     return ap.parse_args()
@@ -209,12 +215,16 @@ def main():
     w = wl.CONFIGS[args.config]
     if args.layers or args.batch:
         w = wl.small(w, n_layers=args.layers or w.n_layers, batch=args.batch or w.batch)
+    if args.spec_fidelity is not None:
+        w = wl.small(w, spec_fidelity=args.spec_fidelity)
     L, B, K, W = w.n_layers, w.batch, args.steps, max(args.warmup, 0)
     hbm_peak, peak_src = measured_peaks()
 
     compute = torch.cuda.Stream()
     copy = torch.cuda.Stream(priority=0)
-    urgent = torch.cuda.Stream(priority=-1) if args.correct_misses else None
+    urgent = None
+    if args.correct_misses:
+        urgent = copy if args.urgent_fifo else torch.cuda.Stream(priority=-1)
     gm = dd.DD_GATHER_BULK if args.gather_mode == "bulk" else dd.DD_GATHER_LOADS
     ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                      forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
@@ -353,6 +363,8 @@ def main():
     if miss is not None:
         line["miss_correction"] = {"missing_pages": miss[0], "selected_pages": miss[1],
                                    "miss_rate": miss[0] / max(1, miss[1]),
+                                   "urgent_queue": "fifo behind the prefetches" if args.urgent_fifo else "own high-priority stream",
+                                   "spec_fidelity": w.spec_fidelity,
                                    "extra_link_bytes_per_layer": miss[0] * w.page_bytes / max(1, (W + K) * L),
                                    "note": "attention runs over the set selected from the current token; the pages the "
                                            "prediction missed cross the link on the urgent stream (counts include warm-up)"}

@@ -44,6 +44,7 @@ class Workload:
     topic_gain: float = math.sqrt(HEAD_DIM)
     planted_noise: float = 0.25
     query_topic: float = 0.5
+    spec_fidelity: float = 0.97   # correlation of step t's speculated query with step t+1's current query
     window_tokens: int = 64
     window_frac: float = 0.10
     window_norm: float = 2.0
@@ -131,9 +132,18 @@ def queries(w: Workload, step: int, layer: int, device="cpu") -> torch.Tensor:
             g = _gen("cpu", w.seed, 13, step + 1, layer)
             q = torch.randn(q.shape, generator=g, dtype=torch.float32).to(torch.bfloat16)
         return q.to(device)
-    g = _gen("cpu", w.seed, 17, step + 1, layer)
     B, Hq, d, G = w.batch, w.n_q_heads, w.head_dim, w.n_q_heads // w.n_kv_heads
-    noise = torch.randn(B, 2, Hq, d, generator=g, dtype=torch.float32)
+
+    def spec_noise(t):
+        return torch.randn(B, 1, Hq, d, generator=_gen("cpu", w.seed, 17, t + 1, layer), dtype=torch.float32)
+
+    # The speculated token of a step stands for the next step's real token (Sec. 4.1): the current token of
+    # step t is the speculated token of step t-1 seen through noise. The first step's current token pairs
+    # with the priming query (step -1).
+    rho = w.spec_fidelity
+    fresh = torch.randn(B, 1, Hq, d, generator=_gen("cpu", w.seed, 31, step + 1, layer), dtype=torch.float32)
+    cur = rho * spec_noise(step - 1) + math.sqrt(1.0 - rho * rho) * fresh if step >= 0 else fresh
+    noise = torch.cat([cur, spec_noise(step)], dim=1)
     if w.structure == "iid" or w.structure == "windows":
         return noise.to(torch.bfloat16).to(device)
     u = torch.stack([topic(w, layer, b) for b in range(B)])            # [B, Hkv, d]

@@ -32,11 +32,15 @@ def _inputs(w, S, ragged=True):
     return store, lms, ctx_len, npg, q_init, q_steps
 
 
-def _run(dd, w, S, inp, depth, mode=0, read_idx=True):
+def _run(dd, w, S, inp, depth, mode=0, read_idx=True, one_stream=False):
     store, lms, ctx_len, npg, q_init, q_steps = inp
     L, B = w.n_layers, w.batch
+    streams = {}
+    if one_stream:                # fully synchronous schedule: gathers, attention and selection on one stream
+        st = torch.cuda.Stream()
+        streams = dict(compute_stream=st, copy_stream=st)
     c = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
-                   forced_recent_pages=w.forced_recent_pages, ring_depth=depth, gather_mode=mode)
+                   forced_recent_pages=w.forced_recent_pages, ring_depth=depth, gather_mode=mode, **streams)
     lm_dev = [x.cuda() for x in lms]
     c.bind(lm_dev, store, npg.cuda(), ctx_len.cuda())
     c.prime(q_init.cuda())
@@ -77,10 +81,12 @@ def test_chain_matches_oracle_and_is_invariant_to_ring_depth_and_engine(dd):
                                       npg.numpy(), ctx_len.numpy(), w.k_pages, T, w.forced_recent_pages)
     if np.array_equal(o_idxs[:S], idxs):
         check_attention(outs, o_outs)
-    # same bits whatever the ring depth, the gather engine, and with no host reads in between
-    for depth, mode, read in [(3, 0, True), (4, 0, False), (2, 1, False), (2, 0, False)]:
-        o2, i2 = _run(dd, w, S, inp, depth=depth, mode=mode, read_idx=read)
-        assert np.array_equal(raw16(o2), raw16(outs)), (depth, mode)
+    # same bits whatever the ring depth, the gather engine, with no host reads in between, and with the whole
+    # schedule serialised on a single stream
+    for depth, mode, read, one in [(3, 0, True, False), (4, 0, False, False), (2, 1, False, False), (2, 0, False, False),
+                                   (2, 0, False, True)]:
+        o2, i2 = _run(dd, w, S, inp, depth=depth, mode=mode, read_idx=read, one_stream=one)
+        assert np.array_equal(raw16(o2), raw16(outs)), (depth, mode, one)
         if read:
             assert np.array_equal(i2, idxs)
 
