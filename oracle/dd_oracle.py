@@ -45,6 +45,7 @@ __all__ = [
     "select_topk",
     "gather_kv",
     "sparse_decode_attn",
+    "sparse_decode_attn_causal",
     "decode_chain",
     "correct_misses",
     "decode_chain_corrected",
@@ -214,6 +215,42 @@ def sparse_decode_attn(q: np.ndarray, slot: np.ndarray, idx: np.ndarray, ctx_len
                         weights[b, t, h] = w
     if return_weights:
         return out, lse, weights
+    return out, lse
+
+
+def sparse_decode_attn_causal(q: np.ndarray, slot: np.ndarray, idx: np.ndarray, ctx_len: np.ndarray,
+                              page_tokens: int, k_new: np.ndarray, v_new: np.ndarray):
+    """Attention of the step's tokens over the gathered set plus the step's own new KV entries, with the
+    dual-token mask (Sec. 5.2 "Dual-token decoding": output token and speculated token of a request are
+    concatenated along the sequence, and the output token must not see the speculated token).
+
+    Query token t (0 = output token, 1 = speculated token) sees every valid gathered token and the new
+    entries j <= t, i.e. itself and the tokens before it. k_new, v_new [B, Tq, Hkv, d] are the keys and
+    values of the step's tokens (context positions ctx_len[b] + j). Returns (out [B, Tq, Hq, d], lse)."""
+    q = np.asarray(q, dtype=np.float64)
+    slot = np.asarray(slot, dtype=np.float64)
+    k_new = np.asarray(k_new, dtype=np.float64)
+    v_new = np.asarray(v_new, dtype=np.float64)
+    B, Tq, Hq, d = q.shape
+    Hkv = slot.shape[1]
+    G = Hq // Hkv
+    T = page_tokens
+    out = np.zeros((B, Tq, Hq, d), dtype=np.float64)
+    lse = np.zeros((B, Tq, Hq), dtype=np.float64)
+    for b in range(B):
+        for g in range(Hkv):
+            pos = (idx[b, g].astype(np.int64)[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+            valid = pos < int(ctx_len[b])
+            for t in range(Tq):
+                keys = np.concatenate([slot[b, g, 0][valid], k_new[b, :t + 1, g]], axis=0)
+                vals = np.concatenate([slot[b, g, 1][valid], v_new[b, :t + 1, g]], axis=0)
+                for h in range(g * G, (g + 1) * G):
+                    z = keys @ q[b, t, h] / np.sqrt(float(d))
+                    m = z.max()
+                    e = np.exp(z - m)
+                    den = e.sum()
+                    out[b, t, h] = (e / den) @ vals
+                    lse[b, t, h] = m + np.log(den)
     return out, lse
 
 

@@ -369,3 +369,46 @@ def test_corrected_chain_equals_attention_over_the_true_sets():
     outs2, pred2, _, _ = orc.decode_chain_corrected(q_init + 3.0, q_steps, lm, kv, npg, ctx, k, T)
     assert not np.array_equal(pred[0], pred2[0])
     np.testing.assert_allclose(outs, outs2, rtol=1e-12, atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- dual-token causal tail
+def test_causal_tail_equals_dense_causal_attention_over_the_extended_sequence():
+    """Full budget: context of n tokens, then the output token, then the speculated token. The result must be
+    dense attention over [context, new tokens] with the causal mask, computed here by torch SDPA with an
+    explicit boolean mask (the output token does not see the speculated token; both see the whole context)."""
+    rng = np.random.default_rng(30)
+    B, Tq, Hq, Hkv, P, T, d = 2, 2, 8, 2, 5, 4, 16
+    q = rng.standard_normal((B, Tq, Hq, d))
+    kv = rng.standard_normal((B, Hkv, P, 2, T, d))
+    k_new = rng.standard_normal((B, Tq, Hkv, d))
+    v_new = rng.standard_normal((B, Tq, Hkv, d))
+    ident = np.tile(np.arange(P, dtype=np.int32), (B, Hkv, 1))
+    ctx = np.array([P * T, P * T - 2])
+    out, lse = orc.sparse_decode_attn_causal(q, orc.gather_kv(kv, ident), ident, ctx, T, k_new, v_new)
+    G = Hq // Hkv
+    for b in range(B):
+        n = int(ctx[b])
+        K = np.concatenate([kv[b, :, :, 0].reshape(Hkv, P * T, d)[:, :n], k_new[b].transpose(1, 0, 2)], axis=1)
+        V = np.concatenate([kv[b, :, :, 1].reshape(Hkv, P * T, d)[:, :n], v_new[b].transpose(1, 0, 2)], axis=1)
+        Kt = torch.from_numpy(K).repeat_interleave(G, dim=0)
+        Vt = torch.from_numpy(V).repeat_interleave(G, dim=0)
+        Q = torch.from_numpy(q[b]).permute(1, 0, 2)
+        mask = torch.ones(Tq, n + Tq, dtype=torch.bool)
+        mask[0, n + 1] = False                                        # output token does not see the speculated one
+        ref = torch.nn.functional.scaled_dot_product_attention(Q, Kt, Vt, attn_mask=mask).permute(1, 0, 2).numpy()
+        np.testing.assert_allclose(out[b], ref, rtol=1e-10, atol=1e-12)
+    # the speculated token's own entry matters to it and not to the output token
+    k2, v2 = k_new.copy(), v_new.copy()
+    k2[:, 1] += 1.0
+    v2[:, 1] -= 2.0
+    out2, _ = orc.sparse_decode_attn_causal(q, orc.gather_kv(kv, ident), ident, ctx, T, k2, v2)
+    assert np.array_equal(out2[:, 0], out[:, 0]) and not np.allclose(out2[:, 1], out[:, 1])
+    # merging by log-sum-exp: the tail result is the lse-weighted mix of the set-only result and the tail's own
+    o_set, lse_set = orc.sparse_decode_attn(q, orc.gather_kv(kv, ident), ident, ctx, T)
+    b, t, h = 1, 1, 5
+    g = h // G
+    z_tail = k_new[b, :t + 1, g] @ q[b, t, h] / math.sqrt(d)
+    w_set = math.exp(lse_set[b, t, h] - lse[b, t, h])
+    w_tail = np.exp(z_tail - lse[b, t, h])
+    np.testing.assert_allclose(out[b, t, h], w_set * o_set[b, t, h] + w_tail @ v_new[b, :t + 1, g], rtol=1e-10)
+    assert abs(w_set + w_tail.sum() - 1.0) < 1e-12
