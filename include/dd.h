@@ -186,6 +186,18 @@ int dd_prime(dd_ctx* ctx, const void* q_init);
  *   out  dev bf16 [B][Tq][Hq][d], written */
 int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out);
 
+/* ---- dual-token causal tail (Sec. 5.2 "Dual-token decoding") ----------------------------------------- */
+
+/* The same attention with the step's own new KV entries appended: the output token and the speculated token
+ * of a request are concatenated along the sequence, and the output token must not see the speculated token.
+ * Query token t sees every valid gathered token and the new entries j <= t (itself and the tokens before it).
+ *   k_new, v_new  dev bf16 [B][Tq][Hkv][d]: keys and values of the step's tokens (token 0 = output token)
+ * Everything else as in dd_sparse_decode_attn / dd_decode_layer_step. out_lse includes the new entries. */
+int dd_sparse_decode_attn_causal(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len,
+                                 const void* k_new, const void* v_new, void* out, float* out_lse, void* stream);
+int dd_decode_layer_step_causal(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new,
+                                const void* v_new, void* out);
+
 /* Device address of the predicted index set [B][Hkv][k] prefetched for (step parity, layer). No copy. */
 int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx);
 

@@ -33,7 +33,7 @@ EXPORTS = [
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
-    "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
+    "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
 ]
 
 
@@ -82,6 +82,8 @@ def _load() -> C.CDLL:
     lib.dd_prime.argtypes = [vp, vp]
     lib.dd_decode_layer_step.argtypes = [vp, ip, ip, vp, vp]
     lib.dd_get_indices.argtypes = [vp, ip, ip, C.POINTER(vp)]
+    lib.dd_sparse_decode_attn_causal.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp, vp]
+    lib.dd_decode_layer_step_causal.argtypes = [vp, ip, ip, vp, vp, vp, vp]
     lib.dd_diff_indices.argtypes = [vp, vp, vp, ip, vp, vp]
     lib.dd_fetch_missing_from_host.argtypes = [vp, vp, ip, vp]
     lib.dd_get_merged_indices.argtypes = [vp, ip, C.POINTER(vp)]
@@ -228,6 +230,13 @@ class Context:
     def sparse_decode_attn(self, q, slot, idx, ctx_len, out, out_lse=None, stream=None):
         self._check(lib.dd_sparse_decode_attn(self._h, _ptr(q), slot, _ptr(idx), _ptr(ctx_len), _ptr(out),
                                               _ptr(out_lse), _stream(stream)))
+
+    def sparse_decode_attn_causal(self, q, slot, idx, ctx_len, k_new, v_new, out, out_lse=None, stream=None):
+        self._check(lib.dd_sparse_decode_attn_causal(self._h, _ptr(q), slot, _ptr(idx), _ptr(ctx_len), _ptr(k_new),
+                                                     _ptr(v_new), _ptr(out), _ptr(out_lse), _stream(stream)))
+
+    def decode_layer_step_causal(self, step, layer, q, k_new, v_new, out):
+        self._check(lib.dd_decode_layer_step_causal(self._h, step, layer, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out)))
 
     def bind(self, landmarks_per_layer, host_kv_per_layer, n_pages, ctx_len):
         L = self.cfg.n_layers

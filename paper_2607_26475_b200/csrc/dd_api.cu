@@ -470,7 +470,8 @@ extern "C" int dd_prime(dd_ctx* ctx, const void* q_init) {
   return DD_OK;
 }
 
-extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out) {
+static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new, const void* v_new,
+                              void* out) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_decode_layer_step: ctx is NULL");
   if (!ctx->primed) return dd_fail(ctx, DD_ERR_STATE, "dd_decode_layer_step: call dd_bind and dd_prime first");
   const dd_config& c = ctx->cfg;
@@ -481,6 +482,8 @@ extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void
                    ctx->next_call % c.n_layers, step, layer);
   DD_TRY(dd_check_dev(ctx, q, "q"));
   DD_TRY(dd_check_dev(ctx, out, "out"));
+  if (k_new) DD_TRY(dd_check_dev(ctx, k_new, "k_new"));
+  if (k_new) DD_TRY(dd_check_dev(ctx, v_new, "v_new"));
   cudaStream_t cs = (cudaStream_t)c.compute_stream;
   const int slot = (int)(n % c.ring_depth);
 
@@ -507,7 +510,8 @@ extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void
   } else {
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));                  // transfer complete
   }
-  DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, attn_idx, ctx->ctx_len, out, nullptr, cs));
+  DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, attn_idx, ctx->ctx_len, out, nullptr, cs,
+                        k_new, v_new));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
   ctx->released_recorded[slot] = true;
   if (!c.miss_correction) {
@@ -521,6 +525,33 @@ extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void
   DD_TRY(dd_enqueue_gather(ctx, n + ahead));
   ctx->next_call = n + 1;
   return DD_OK;
+}
+
+extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out) {
+  return dd_layer_step_impl(ctx, step, layer, q, nullptr, nullptr, out);
+}
+
+extern "C" int dd_decode_layer_step_causal(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new,
+                                           const void* v_new, void* out) {
+  if (!k_new || !v_new) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_decode_layer_step_causal: k_new / v_new is NULL");
+  return dd_layer_step_impl(ctx, step, layer, q, k_new, v_new, out);
+}
+
+extern "C" int dd_sparse_decode_attn_causal(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len,
+                                            const void* k_new, const void* v_new, void* out, float* out_lse,
+                                            void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_causal: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  DD_TRY(dd_check_dev(ctx, q, "q"));
+  DD_TRY(dd_check_dev(ctx, idx, "idx", 4));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
+  DD_TRY(dd_check_dev(ctx, k_new, "k_new"));
+  DD_TRY(dd_check_dev(ctx, v_new, "v_new"));
+  DD_TRY(dd_check_dev(ctx, out, "out"));
+  if (out_lse) DD_TRY(dd_check_dev(ctx, out_lse, "out_lse", 4));
+  return dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, idx, ctx_len, out, out_lse,
+                        (cudaStream_t)stream, k_new, v_new);
 }
 
 extern "C" int dd_get_indices(dd_ctx* ctx, int step_parity, int layer, const int** dev_idx) {

@@ -70,7 +70,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     const __nv_bfloat16* __restrict__ q, const char* __restrict__ slot, const int* __restrict__ idx,
     const int* __restrict__ ctx_len, __nv_bfloat16* __restrict__ out, float* __restrict__ out_lse,
     float* __restrict__ part_o, float2* __restrict__ part_ml, unsigned int* __restrict__ ticket, int Hkv, int G, int Tq,
-    int k, int n_splits, int pages_per_split, int cluster) {
+    int k, int n_splits, int pages_per_split, int cluster, const __nv_bfloat16* __restrict__ k_new,
+    const __nv_bfloat16* __restrict__ v_new) {
   const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gl = lane >> 2, t = lane & 3;
@@ -111,37 +112,22 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
   float m_run[2] = {-INFINITY, -INFINITY};   // columns n = 2t, 2t+1, log2 domain
   float l_run[2] = {0.f, 0.f};               // partial over this lane's tokens
 
-  const int p_begin = split * pages_per_split;
-  const int p_end = min(k, p_begin + pages_per_split);
-  int j = p_begin + warp;
   uint4 klo[4], khi[4], v[4][2];
-  int page = 0;
-  if (j < p_end) {
-    dd_load_k(kbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
-    dd_load_v(vbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, v);
-    page = idx_bg[j];
-  }
-  while (j < p_end) {
-    const int jn = j + ATTN_WARPS;
-    const bool has_next = jn < p_end;
-    // ---- S^T = K q^T
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+
+  // S^T = K q^T for the page held in klo / khi, scaled to the log2 domain
+  auto qk = [&](float (&acc)[4]) {
+    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
       dd_mma_bf16(acc, klo[kk].x, khi[kk].x, klo[kk].y, khi[kk].y, qf[kk].x, qf[kk].y);
       dd_mma_bf16(acc, klo[kk].z, khi[kk].z, klo[kk].w, khi[kk].w, qf[kk].z, qf[kk].w);
     }
-    // the K fragments are consumed: the next page's K goes into the same registers while this page finishes
-    if (has_next) dd_load_k(kbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
-    const int page_next = has_next ? idx_bg[jn] : 0;
     // acc[0], acc[1]: token gl, columns 2t, 2t+1; acc[2], acc[3]: token gl+8
 #pragma unroll
     for (int i = 0; i < 4; ++i) acc[i] *= scale_log2;
-    if (page * DD_T + DD_T > n_ctx) {            // only the last page of a request can be partial
-      if (page * DD_T + gl >= n_ctx) acc[0] = acc[1] = -INFINITY;
-      if (page * DD_T + gl + 8 >= n_ctx) acc[2] = acc[3] = -INFINITY;
-    }
-    // ---- running soft-max per column
+  };
+  // running soft-max per column, then O^T += V^T P^T with the page held in v
+  auto softmax_pv = [&](float (&acc)[4]) {
     float alpha[2], pr[4];
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
@@ -164,10 +150,10 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     for (int i = 0; i < 8; ++i) {
       o[i][0] *= alpha[0]; o[i][1] *= alpha[1]; o[i][2] *= alpha[0]; o[i][3] *= alpha[1];
     }
-    // ---- P^T as the B operand: tokens {2t, 2t+1} and {2t+8, 2t+9} of column gl
+    // P^T as the B operand: tokens {2t, 2t+1} and {2t+8, 2t+9} of column gl
     const uint32_t pb0 = dd_movmatrix_trans(dd_pack_bf16(pr[0], pr[1]));
     const uint32_t pb1 = dd_movmatrix_trans(dd_pack_bf16(pr[2], pr[3]));
-    // ---- O^T += V^T P^T; MMA tile i has rows gl -> channel 8gl+i and gl+8 -> channel 64+8gl+i
+    // MMA tile i has rows gl -> channel 8gl+i and gl+8 -> channel 64+8gl+i
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int w = i >> 1;
@@ -178,6 +164,61 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
       const uint32_t a3 = __byte_perm(dd_word(v[2][1], w), dd_word(v[3][1], w), sel);
       dd_mma_bf16(o[i], a0, a1, a2, a3, pb0, pb1);
     }
+  };
+
+  // ---- the step's own new KV entries (dual-token causal tail): one extra "page" whose tokens 0..Tq-1 are the
+  // new entries; query token t sees the entries j <= t. Taken by the first warp of the first split.
+  if (k_new != nullptr && split == 0 && warp == 0) {
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      klo[kk] = gl < Tq ? __ldg(reinterpret_cast<const uint4*>(k_new + (((size_t)b * Tq + gl) * Hkv + g) * DD_D) + kk * 4 + t)
+                        : zero;
+      khi[kk] = zero;
+    }
+#pragma unroll
+    for (int tk = 0; tk < 4; ++tk) {
+      const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+        v[tk][c] = tok < Tq ? __ldg(reinterpret_cast<const uint4*>(v_new + (((size_t)b * Tq + tok) * Hkv + g) * DD_D +
+                                                                  c * 64 + gl * 8))
+                            : zero;
+    }
+    float acc[4];
+    qk(acc);
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int n = 2 * t + c;                   // query row: token n / G
+      const bool visible = gl < Tq && n < n_rows && gl <= n / G;
+      if (!visible) acc[c] = -INFINITY;
+      acc[2 + c] = -INFINITY;
+    }
+    softmax_pv(acc);
+  }
+
+  const int p_begin = split * pages_per_split;
+  const int p_end = min(k, p_begin + pages_per_split);
+  int j = p_begin + warp;
+  int page = 0;
+  if (j < p_end) {
+    dd_load_k(kbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
+    dd_load_v(vbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, v);
+    page = idx_bg[j];
+  }
+  while (j < p_end) {
+    const int jn = j + ATTN_WARPS;
+    const bool has_next = jn < p_end;
+    float acc[4];
+    qk(acc);
+    // the K fragments are consumed: the next page's K goes into the same registers while this page finishes
+    if (has_next) dd_load_k(kbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
+    const int page_next = has_next ? idx_bg[jn] : 0;
+    if (page * DD_T + DD_T > n_ctx) {            // only the last page of a request can be partial
+      if (page * DD_T + gl >= n_ctx) acc[0] = acc[1] = -INFINITY;
+      if (page * DD_T + gl + 8 >= n_ctx) acc[2] = acc[3] = -INFINITY;
+    }
+    softmax_pv(acc);
     if (has_next) dd_load_v(vbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, v);
     if (j == p_begin + warp) DD_TRACE_MARK(1);
     page = page_next;
@@ -367,7 +408,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
 // Launch with clusters of `cluster` blocks along x (1 = no cluster attribute needed).
 static cudaError_t dd_attn_launch_raw(cudaStream_t st, int batch, int Hkv, int G, int Tq, int k, int n_splits,
                                       int cluster, const void* q, const char* slot, const int* idx, const int* ctx_len,
-                                      void* out, float* out_lse, float* part_o, float2* part_ml, unsigned int* ticket) {
+                                      void* out, float* out_lse, float* part_o, float2* part_ml, unsigned int* ticket,
+                                      const void* k_new = nullptr, const void* v_new = nullptr) {
   const int pps = (k + n_splits - 1) / n_splits;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_splits, Hkv, batch);
@@ -382,15 +424,16 @@ static cudaError_t dd_attn_launch_raw(cudaStream_t st, int batch, int Hkv, int G
   cfg.attrs = attr;
   cfg.numAttrs = cluster > 1 ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, dd_attn_kernel, (const __nv_bfloat16*)q, slot, idx, ctx_len, (__nv_bfloat16*)out,
-                            out_lse, part_o, part_ml, ticket, Hkv, G, Tq, k, n_splits, pps, cluster);
+                            out_lse, part_o, part_ml, ticket, Hkv, G, Tq, k, n_splits, pps, cluster,
+                            (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
 }
 
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
-                   float* out_lse, cudaStream_t st) {
+                   float* out_lse, cudaStream_t st, const void* k_new, const void* v_new) {
   const dd_config& c = ctx->cfg;
   DD_CUDA_TRY(ctx, dd_attn_launch_raw(st, c.batch, c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, ctx->attn_splits,
                                       ctx->attn_cluster, q, slot, idx, ctx_len, out, out_lse, ctx->attn_part_o,
-                                      ctx->attn_part_ml, ctx->attn_ticket));
+                                      ctx->attn_part_ml, ctx->attn_ticket, k_new, v_new));
   return DD_OK;
 }
 

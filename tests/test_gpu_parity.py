@@ -274,3 +274,40 @@ def test_full_budget_equals_dense_attention(dd):
         ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V).permute(1, 0, 2).numpy()
         check_attention(out[b], ref)
     c.close()
+
+
+@pytest.mark.parametrize("B,P,k,ctx_len,Tq,splits,G", [
+    (2, 100, 23, [1600, 1589], 2, 0, 4),
+    (2, 100, 23, [1600, 1589], 2, 5, 4),           # several clusters: the tail enters through the global merge
+    (1, 256, 16, [4096], 2, 1, 4),
+    (2, 64, 8, [1024, 1001], 1, 2, 8),             # one query token: it sees only its own new entry
+    (3, 300, 128, [4800, 4799, 2049], 2, 0, 2),
+])
+def test_attention_with_causal_tail_matches_oracle(dd, B, P, k, ctx_len, Tq, splits, G):
+    Hq = HKV * G
+    g = torch.Generator().manual_seed(B * 77 + k)
+    kv = torch.randn(B, HKV, P, 2, T, D, generator=g).to(torch.bfloat16).pin_memory()
+    q = torch.randn(B, Tq, Hq, D, generator=g).to(torch.bfloat16)
+    k_new = torch.randn(B, Tq, HKV, D, generator=g).to(torch.bfloat16)
+    v_new = (torch.randn(B, Tq, HKV, D, generator=g) * 3).to(torch.bfloat16)
+    k_new[0, 0, 0] = (4.0 * q[0, 0, 0].float()).to(torch.bfloat16)     # one new key that dominates its row
+    cl = torch.tensor(ctx_len, dtype=torch.int32)
+    idx = torch.empty((B, HKV, k), dtype=torch.int32)
+    for b in range(B):
+        last = (int(cl[b]) - 1) // T
+        for h in range(HKV):
+            s = torch.randperm(last, generator=g)[:k - 1].tolist() + [last]
+            idx[b, h] = torch.tensor(sorted(s), dtype=torch.int32)
+    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_q_tokens=Tq, attn_splits=splits)
+    c.gather_kv_from_host(kv, idx.cuda(), None, 0)
+    out = torch.full((B, Tq, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros((B, Tq, Hq), dtype=torch.float32, device="cuda")
+    c.sparse_decode_attn_causal(q.cuda(), 0, idx.cuda(), cl.cuda(), k_new.cuda(), v_new.cuda(), out, lse)
+    assert c.device_error() == (0, 0)
+    slot = orc.gather_kv(f32(kv), idx.numpy())
+    want, want_lse = orc.sparse_decode_attn_causal(f32(q), slot, idx.numpy(), cl.numpy(), T, f32(k_new), f32(v_new))
+    check_attention(out, want)
+    np.testing.assert_allclose(lse.cpu().numpy(), want_lse, atol=2e-3, rtol=1e-4)
+    base, _ = orc.sparse_decode_attn(f32(q), slot, idx.numpy(), cl.numpy(), T)
+    assert np.abs(want - base).max() > 0.1          # the tail matters in this case
+    c.close()

@@ -108,6 +108,36 @@ def test_single_layer_model_with_a_deeper_ring(dd):
             check_selection(idxs[t, 0, 0, h], sc[0][h], w.k_pages, 0)
 
 
+def test_layer_step_with_causal_tail(dd):
+    """The pipelined step with the tokens' own new KV entries appended (output token first, then the
+    speculated token, which also sees the output token's entry)."""
+    S = 2
+    w = wl.small(wl.CONFIGS[2], n_layers=2, batch=2, ctx=16 * 70, budget=16 * 9)
+    store, lms, ctx_len, npg, q_init, q_steps = _inputs(w, S)
+    g = torch.Generator().manual_seed(5)
+    k_new = torch.randn(S, w.n_layers, w.batch, 2, HKV, D, generator=g).to(torch.bfloat16)
+    v_new = torch.randn(S, w.n_layers, w.batch, 2, HKV, D, generator=g).to(torch.bfloat16)
+    c = dd.Context(n_layers=w.n_layers, batch=w.batch, max_pages=w.n_pages, k_pages=w.k_pages)
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qd, kd, vd = q_steps.cuda(), k_new.cuda(), v_new.cuda()
+    outs = torch.zeros_like(qd)
+    idxs = []
+    for t in range(S):
+        idxs.append(torch.stack([c.get_indices(t & 1, l) for l in range(w.n_layers)]).cpu().numpy())
+        for l in range(w.n_layers):
+            c.decode_layer_step_causal(t, l, qd[t, l], kd[t, l], vd[t, l], outs[t, l])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    for t in range(S):
+        for l in range(w.n_layers):
+            slot = orc.gather_kv(f32(store[l]), idxs[t][l])
+            want, _ = orc.sparse_decode_attn_causal(f32(q_steps[t, l]), slot, idxs[t][l], ctx_len.numpy(), T,
+                                                    f32(k_new[t, l]), f32(v_new[t, l]))
+            check_attention(outs[t, l], want)
+    c.close()
+
+
 def test_call_order_is_checked(dd):
     w = wl.small(wl.CONFIGS[2], n_layers=2, batch=1, ctx=16 * 40, budget=16 * 4)
     inp = _inputs(w, 1, ragged=False)
