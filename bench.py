@@ -59,6 +59,7 @@ def parse_args():
     ap.add_argument("--spec-fidelity", type=float, default=None,
                     help="override the generator's correlation between a step's speculated query and the next "
                          "step's current query (lower = more prediction misses)")
+    ap.add_argument("--ragged", action="store_true", help="unequal context lengths per request (second workload shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
     return ap.parse_args()
@@ -231,7 +232,7 @@ def main():
                      gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy,
                      miss_correction=args.correct_misses, urgent_stream=urgent)
     budget = replicas.host_budget_per_rank(available_host_bytes(), world)
-    store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, host_budget_bytes=budget,
+    store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, ragged=args.ragged, host_budget_bytes=budget,
                       log=log if rank == 0 else None)
     store.bind(ctx)
     if rank == 0:
@@ -345,7 +346,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "batch": B, "ctx": w.ctx, "budget": w.budget, "layers": L,
                    "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "gather_mode": args.gather_mode,
+                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "gather_mode": args.gather_mode,
                    "host_store_gib": store.host_bytes / 2**30, "phys_layers": store.n_phys,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2: each layer streams its own 32 MiB of landmarks and 64 MiB of "

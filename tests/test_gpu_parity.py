@@ -311,3 +311,49 @@ def test_attention_with_causal_tail_matches_oracle(dd, B, P, k, ctx_len, Tq, spl
     base, _ = orc.sparse_decode_attn(f32(q), slot, idx.numpy(), cl.numpy(), T)
     assert np.abs(want - base).max() > 0.1          # the tail matters in this case
     c.close()
+
+
+def test_select_precondition_violation_is_reported_and_stays_in_range(dd):
+    """A request with fewer pages than the budget violates k <= n_pages: no trap, the error word is set, and the
+    indices written stay inside the request (the valid pages first, then the last valid page repeated)."""
+    B, P, k = 2, 64, 20
+    g = torch.Generator().manual_seed(2)
+    lm = torch.randn(B, HKV, P, D, generator=g).to(torch.bfloat16).cuda()
+    q = torch.randn(B, 2, HQ, D, generator=g).to(torch.bfloat16).cuda()
+    for mode in (0, 1):
+        c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, select_mode=mode)
+        idx = torch.full((B, HKV, k), -1, dtype=torch.int32, device="cuda")
+        c.select_topk(q, 1, lm, torch.tensor([64, 7], dtype=torch.int32).cuda(), idx)
+        code, detail = c.device_error()
+        assert (code, detail) == (dd.DD_ERR_INDEX_RANGE, 7)
+        got = idx.cpu().numpy()
+        assert np.all(np.diff(got[0], axis=-1) > 0)                      # the healthy request is unaffected
+        assert all(got[1, h].tolist() == list(range(7)) + [6] * (k - 7) for h in range(HKV))
+        # a request that claims more pages than the layout holds is clamped to the layout
+        c.select_topk(q, 1, lm, torch.tensor([64, 1000], dtype=torch.int32).cuda(), idx)
+        assert c.device_error() == (dd.DD_ERR_INDEX_RANGE, 1000)
+        assert idx.max().item() < P and idx.min().item() >= 0
+        c.close()
+
+
+def test_smallest_geometry(dd):
+    """One request, one KV head, one query head, one query token, one page selected out of one."""
+    kv = torch.randn(1, 1, 1, 2, T, D).to(torch.bfloat16).pin_memory()
+    q = torch.randn(1, 1, 1, D).to(torch.bfloat16)
+    cl = torch.tensor([11], dtype=torch.int32)
+    npg = torch.tensor([1], dtype=torch.int32)
+    c = dd.Context(n_layers=1, batch=1, max_pages=1, k_pages=1, n_q_heads=1, n_kv_heads=1, n_q_tokens=1)
+    lm = torch.empty((1, 1, 1, D), dtype=torch.bfloat16, device="cuda")
+    c.build_landmarks(kv, cl.cuda(), lm)
+    idx = torch.full((1, 1, 1), 9, dtype=torch.int32, device="cuda")
+    c.select_topk(q.cuda(), 0, lm, npg.cuda(), idx)
+    c.gather_kv_from_host(kv, idx, npg.cuda(), 0)
+    out = torch.empty((1, 1, 1, D), dtype=torch.bfloat16, device="cuda")
+    c.sparse_decode_attn(q.cuda(), 0, idx, cl.cuda(), out)
+    assert c.device_error() == (0, 0)
+    assert idx.item() == 0
+    assert np.array_equal(f32(lm), orc.build_landmarks(f32(kv[:, :, :, 0]), cl.numpy()))
+    slot = orc.gather_kv(f32(kv), idx.cpu().numpy())
+    want, _ = orc.sparse_decode_attn(f32(q), slot, idx.cpu().numpy(), cl.numpy(), T)
+    check_attention(out, want)
+    c.close()
