@@ -66,32 +66,40 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     return bits.astype(np.uint32).view(np.float32).reshape(a.shape)
 
 
-def build_landmarks(k_pages: np.ndarray, ctx_len: np.ndarray) -> np.ndarray:
-    """Landmark of a page = mean of its valid keys (Sec. 2.2: chunks of adjacent
+def build_landmarks(k_pages: np.ndarray, ctx_len: np.ndarray, chunk_tokens: int | None = None) -> np.ndarray:
+    """Landmark of a chunk = mean of its valid keys (Sec. 2.2: chunks of adjacent
     KV entries with compressed landmarks; Sec. 4.1: built before decoding, fixed).
 
-    k_pages [B, Hkv, P, T, d] bf16-valued; ctx_len [B] tokens. A page with no
-    valid token gets a zero landmark (it is never scored). The storage format is
-    part of the definition: sum in fp32 in token order, divide in fp32, round to
-    bf16, so that the same bits can be produced by any implementation.
+    k_pages [B, Hkv, P, T, d] bf16-valued; ctx_len [B] tokens. A chunk is
+    `chunk_tokens` consecutive tokens of a page (default: the whole page, T);
+    the result is [B, Hkv, P * T / chunk_tokens, d], chunks of a page adjacent.
+    A chunk with no valid token gets a zero landmark (it is never scored). The
+    storage format is part of the definition: sum in fp32 in token order, divide
+    in fp32, round to bf16, so that the same bits can be produced by any
+    implementation.
     """
     k_pages = np.asarray(k_pages, dtype=np.float32)
     B, Hkv, P, T, d = k_pages.shape
-    out = np.zeros((B, Hkv, P, d), dtype=np.float32)
+    c = T if chunk_tokens is None else int(chunk_tokens)
+    assert T % c == 0
+    toks = k_pages.reshape(B, Hkv, P * T, d)
+    n_chunks = P * T // c
+    out = np.zeros((B, Hkv, n_chunks, d), dtype=np.float32)
     for b in range(B):
         n_tok = int(ctx_len[b])
-        for p in range(P):
-            cnt = min(T, n_tok - p * T)
+        for ch in range(n_chunks):
+            cnt = min(c, n_tok - ch * c)
             if cnt <= 0:
                 continue
             acc = np.zeros((Hkv, d), dtype=np.float32)
             for i in range(cnt):
-                acc = acc + k_pages[b, :, p, i, :]
-            out[b, :, p, :] = acc / np.float32(cnt)
+                acc = acc + toks[b, :, ch * c + i, :]
+            out[b, :, ch, :] = acc / np.float32(cnt)
     return round_to_bf16(out)
 
 
-def page_scores(q_tok: np.ndarray, lm: np.ndarray, n_pages: int, group_reduce: str = "softmax_max"):
+def page_scores(q_tok: np.ndarray, lm: np.ndarray, n_pages: int, group_reduce: str = "softmax_max",
+                chunks_per_page: int = 1, n_chunks: int | None = None):
     """Scores of one request's pages for every KV head (Sec. 4.1).
 
     q_tok [Hq, d] (the scoring token's per-head queries), lm [Hkv, P, d].
@@ -103,7 +111,21 @@ def page_scores(q_tok: np.ndarray, lm: np.ndarray, n_pages: int, group_reduce: s
 
     `group_reduce` other than "softmax_max" exists only to show sensitivity to
     the reading ("logit_max", "logit_mean"); the contract is "softmax_max".
+
+    With finer landmarks (chunks_per_page = R > 1, lm [Hkv, P * R, d], the first
+    n_chunks chunks of the request exist) the soft-max runs over the existing
+    chunks and a page takes the maximum over its chunks as well:
+      score[g, p] = max_{h in group g, r < R} exp(s[h, p * R + r] - lse[h]);
+    s and lse are then returned per chunk.
     """
+    if chunks_per_page != 1:
+        R = int(chunks_per_page)
+        nc = int(n_chunks)
+        assert (n_pages - 1) * R < nc <= n_pages * R
+        chunk_score, s, lse = page_scores(q_tok, lm, nc, "softmax_max")
+        padded = np.zeros((chunk_score.shape[0], n_pages * R), dtype=np.float64)
+        padded[:, :nc] = chunk_score
+        return padded.reshape(-1, n_pages, R).max(axis=2), s, lse
     q_tok = np.asarray(q_tok, dtype=np.float64)
     lm = np.asarray(lm, dtype=np.float64)
     Hq, d = q_tok.shape
@@ -143,17 +165,20 @@ def topk_pages(score: np.ndarray, k: int, forced_recent: int = 0) -> np.ndarray:
 
 
 def select_topk(q_tok: np.ndarray, lm: np.ndarray, n_pages: np.ndarray, k: int,
-                forced_recent: int = 0, group_reduce: str = "softmax_max"):
+                forced_recent: int = 0, group_reduce: str = "softmax_max", chunks_per_page: int = 1,
+                n_chunks: np.ndarray | None = None):
     """Per-KV-head critical set of every request (Sec. 2.2, Sec. 4.1).
 
-    q_tok [B, Hq, d], lm [B, Hkv, P, d], n_pages [B].
+    q_tok [B, Hq, d], lm [B, Hkv, P * chunks_per_page, d], n_pages [B] (and n_chunks [B], the existing
+    chunks of every request, when chunks_per_page > 1).
     Returns (idx [B, Hkv, k] int32 ascending, scores: list of [Hkv, n_pages[b]])."""
     B = q_tok.shape[0]
     Hkv = lm.shape[1]
     idx = np.empty((B, Hkv, k), dtype=np.int32)
     scores = []
     for b in range(B):
-        sc, _, _ = page_scores(q_tok[b], lm[b], int(n_pages[b]), group_reduce)
+        sc, _, _ = page_scores(q_tok[b], lm[b], int(n_pages[b]), group_reduce, chunks_per_page,
+                               None if n_chunks is None else int(n_chunks[b]))
         scores.append(sc)
         for g in range(Hkv):
             idx[b, g] = topk_pages(sc[g], k, forced_recent)

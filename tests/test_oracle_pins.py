@@ -412,3 +412,53 @@ def test_causal_tail_equals_dense_causal_attention_over_the_extended_sequence():
     w_tail = np.exp(z_tail - lse[b, t, h])
     np.testing.assert_allclose(out[b, t, h], w_set * o_set[b, t, h] + w_tail @ v_new[b, :t + 1, g], rtol=1e-10)
     assert abs(w_set + w_tail.sum() - 1.0) < 1e-12
+
+
+# ----------------------------------------------------------------------------- finer landmarks
+def test_chunk_landmarks_and_chunked_page_scores():
+    rng = np.random.default_rng(40)
+    B, Hkv, Hq, P, T, d, c = 1, 2, 4, 6, 8, 16, 2
+    R = T // c
+    ctx = np.array([P * T - 3])                                  # last chunk of the last page is missing, one is partial
+    keys = orc.round_to_bf16(rng.standard_normal((B, Hkv, P, T, d)).astype(np.float32))
+    lm_c = orc.build_landmarks(keys, ctx, chunk_tokens=c)
+    assert lm_c.shape == (B, Hkv, P * R, d)
+    toks = keys.reshape(B, Hkv, P * T, d).astype(np.float64)
+    for ch in range(P * R):
+        lo, hi = ch * c, min((ch + 1) * c, int(ctx[0]))
+        want = toks[0, :, lo:hi].mean(axis=1) if hi > lo else np.zeros((Hkv, d))
+        assert np.all(np.abs(lm_c[0, :, ch] - want) <= np.maximum(np.abs(want), 1e-30) * 2.0 ** -8)
+    assert np.all(lm_c[0, :, -1] == 0.0)
+    # whole-page chunks are the page landmarks, bit for bit
+    assert np.array_equal(orc.build_landmarks(keys, ctx, chunk_tokens=T), orc.build_landmarks(keys, ctx))
+    # chunked page score = brute force over chunks: soft-max over the existing chunks, max over heads and chunks
+    q = rng.standard_normal((Hq, d))
+    n_chunks = -(-int(ctx[0]) // c)
+    score, s, lse = orc.page_scores(q, lm_c[0], P, chunks_per_page=R, n_chunks=n_chunks)
+    G = Hq // Hkv
+    for g in range(Hkv):
+        for p in range(P):
+            best = 0.0
+            for h in range(g * G, (g + 1) * G):
+                z = [sum(q[h, x] * lm_c[0, g, ch, x] for x in range(d)) / math.sqrt(d) for ch in range(n_chunks)]
+                den = sum(math.exp(v) for v in z)
+                for r in range(R):
+                    ch = p * R + r
+                    if ch < n_chunks:
+                        best = max(best, math.exp(z[ch]) / den)
+            assert abs(score[g, p] - best) <= 1e-12 * best
+    # R = 1 is the page-level definition
+    lm_p = orc.build_landmarks(keys, ctx)
+    a, _, _ = orc.page_scores(q, lm_p[0], P)
+    b2, _, _ = orc.page_scores(q, lm_p[0], P, chunks_per_page=1)
+    assert np.array_equal(a, b2)
+    # one-token chunks: a page scores as its best token does
+    lm_1 = orc.build_landmarks(keys, ctx, chunk_tokens=1)
+    sc1, _, _ = orc.page_scores(q[:2], lm_1[0][:1], P, chunks_per_page=T, n_chunks=int(ctx[0]))
+    logits = toks[0, 0, :int(ctx[0])] @ q[0] / math.sqrt(d)
+    prob = np.exp(logits - logits.max()); prob /= prob.sum()
+    logits1 = toks[0, 0, :int(ctx[0])] @ q[1] / math.sqrt(d)
+    prob1 = np.exp(logits1 - logits1.max()); prob1 /= prob1.sum()
+    both = np.maximum(prob, prob1)
+    pad = np.zeros(P * T); pad[:int(ctx[0])] = both
+    np.testing.assert_allclose(sc1[0], pad.reshape(P, T).max(axis=1), rtol=1e-10)
