@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--spec-fidelity", type=float, default=None,
                     help="override the generator's correlation between a step's speculated query and the next "
                          "step's current query (lower = more prediction misses)")
+    ap.add_argument("--landmark-chunk", type=int, default=0,
+                    help="tokens per landmark: 0/16 = one per page (default), 8/4/2/1 = several per page")
     ap.add_argument("--ragged", action="store_true", help="unequal context lengths per request (second workload shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
@@ -234,7 +236,7 @@ def main():
     ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                      forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
                      gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy,
-                     miss_correction=args.correct_misses, urgent_stream=urgent)
+                     miss_correction=args.correct_misses, urgent_stream=urgent, landmark_chunk_tokens=args.landmark_chunk)
     budget = replicas.host_budget_per_rank(available_host_bytes(), world)
     store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, ragged=args.ragged, host_budget_bytes=budget,
                       log=log if rank == 0 else None)
@@ -350,7 +352,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "batch": B, "ctx": w.ctx, "budget": w.budget, "layers": L,
                    "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "gather_mode": args.gather_mode,
+                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "landmark_chunk_tokens": args.landmark_chunk or w.page_tokens, "gather_mode": args.gather_mode,
                    "host_store_gib": store.host_bytes / 2**30, "phys_layers": store.n_phys,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2: each layer streams its own 32 MiB of landmarks and 64 MiB of "
@@ -452,8 +454,8 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
         total = batch(True)
         return total - (batch(False) if pre else 0.0)
 
-    sel_us = timed(cs, lambda i: ctx.select_topk(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
-                                                 store.n_pages_dev, tmp_idx, None, stream=cs))
+    sel_us = timed(cs, lambda i: ctx.select_topk_chunked(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
+                                                         store.n_pages_dev, store.ctx_len_dev, tmp_idx, None, stream=cs))
     gat_us = timed(xs, lambda i: ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev,
                                                          i % args.ring_depth, stream=xs))
     ctx.gather_kv_from_host(store.kv[0], idx[0], store.n_pages_dev, 0, stream=cs)
@@ -474,11 +476,12 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
             e0.record(cs)
         for l in range(L):
             ctx.sparse_decode_attn(q_dev[0, l], 0, idx[0], store.ctx_len_dev, outs[l], None, stream=cs)
-            ctx.select_topk(q_dev[0, l], 1, store.landmarks[l], store.n_pages_dev, tmp_idx, None, stream=cs)
+            ctx.select_topk_chunked(q_dev[0, l], 1, store.landmarks[l], store.n_pages_dev, store.ctx_len_dev, tmp_idx,
+                                    None, stream=cs)
     e1.record(cs)
     torch.cuda.synchronize()
     compute_only = e0.elapsed_time(e1) * 1e3 / (n_rep * L)
-    lm_bytes = B * w.n_kv_heads * w.n_pages * 256
+    lm_bytes = B * w.n_kv_heads * w.n_pages * 256 * (w.page_tokens // args.landmark_chunk if args.landmark_chunk else 1)
     sel_bytes = float(lm_bytes)           # landmarks once; the fused kernel keeps the logits in shared memory
     gb = w.gathered_bytes_per_layer
     return {

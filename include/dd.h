@@ -74,6 +74,7 @@ typedef struct dd_config {
   void* copy_stream;         /* cudaStream_t used by the pipelined calls for the gather */
   void* ring_mem;            /* optional caller-owned ring of dd_ring_bytes(); NULL = library allocates */
   size_t ring_bytes;         /* size of ring_mem when supplied */
+  int landmark_chunk_tokens; /* tokens summarised by one landmark: 0 or 16 = one per page; 8, 4, 2, 1 = several per page */
   int miss_correction;       /* 1: dd_decode_layer_step repairs prediction misses before attention (needs urgent_stream) */
   void* urgent_stream;       /* cudaStream_t, ideally of higher priority than copy_stream; used for the missing pages */
 } dd_config;
@@ -109,7 +110,9 @@ int dd_sync(dd_ctx* ctx, double timeout_s);
  * round-to-nearest-even to bf16; a page with no valid token gets zeros.
  *   kv_layer   pinned or dev, bf16 [B][Hkv][P][2][T][d] ([..][0] = K, [..][1] = V)
  *   ctx_len    dev int32 [B], tokens per request
- *   landmarks  dev bf16 [B][Hkv][P][d], written */
+ *   landmarks  dev bf16 [B][Hkv][P][d], written
+ * With landmark_chunk_tokens = c < 16 a page has R = 16/c landmarks, one per c consecutive tokens, and the
+ * tensor is [B][Hkv][P*R][d] with the chunks of a page adjacent. */
 int dd_build_landmarks(dd_ctx* ctx, const void* kv_layer, const int* ctx_len, void* landmarks, void* stream);
 
 /* ---- the three kernels of the path ----------------------------------------------------------- */
@@ -131,6 +134,14 @@ int dd_build_landmarks(dd_ctx* ctx, const void* kv_layer, const int* ctx_len, vo
  *   out_scores  dev fp32 [B][Hkv][P] or NULL; score[g,p] for p < n_pages[b], written */
 int dd_select_topk(dd_ctx* ctx, const void* q, int q_token, const void* landmarks, const int* n_pages,
                    int* out_idx, float* out_scores, void* stream);
+
+/* The same selection when pages carry several landmarks (landmark_chunk_tokens < 16; the paper leaves the
+ * chunk size open, Sec. 2.2): the soft-max of a head runs over the chunks that hold at least one token, and a
+ * page's score is the maximum over the group's heads and over the page's chunks. landmarks is
+ * [B][Hkv][P*R][d]; ctx_len (dev int32 [B]) tells which chunks exist. With one landmark per page it equals
+ * dd_select_topk. dd_select_topk itself fails with DD_ERR_INVALID_ARG on a context with several chunks per page. */
+int dd_select_topk_chunked(dd_ctx* ctx, const void* q, int q_token, const void* landmarks, const int* n_pages,
+                           const int* ctx_len, int* out_idx, float* out_scores, void* stream);
 
 /* Gather of the selected pages into a ring slot in attention layout (Sec. 5.3: predicted KV
  * entries are prefetched from host memory; Sec. 5.4 "GPU-side sparse KV assembly": the GPU

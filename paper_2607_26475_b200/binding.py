@@ -33,7 +33,7 @@ EXPORTS = [
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
-    "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
+    "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
 ]
 
 
@@ -46,7 +46,7 @@ class DDConfig(C.Structure):
         ("gather_mode", C.c_int), ("gather_ctas", C.c_int), ("select_mode", C.c_int), ("attn_splits", C.c_int),
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
-        ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
+        ("landmark_chunk_tokens", C.c_int), ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
     ]
 
 
@@ -82,6 +82,7 @@ def _load() -> C.CDLL:
     lib.dd_prime.argtypes = [vp, vp]
     lib.dd_decode_layer_step.argtypes = [vp, ip, ip, vp, vp]
     lib.dd_get_indices.argtypes = [vp, ip, ip, C.POINTER(vp)]
+    lib.dd_select_topk_chunked.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
     lib.dd_sparse_decode_attn_causal.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp, vp]
     lib.dd_decode_layer_step_causal.argtypes = [vp, ip, ip, vp, vp, vp, vp]
     lib.dd_diff_indices.argtypes = [vp, vp, vp, ip, vp, vp]
@@ -147,7 +148,7 @@ class Context:
     def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
                  gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None,
-                 miss_correction=False, urgent_stream=None):
+                 miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
@@ -160,7 +161,7 @@ class Context:
                             forced_recent_pages, n_q_tokens, ring_depth, gather_mode, gather_ctas, select_mode, attn_splits,
                             self.compute_stream.cuda_stream, self.copy_stream.cuda_stream,
                             _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0,
-                            1 if miss_correction else 0,
+                            landmark_chunk_tokens, 1 if miss_correction else 0,
                             self.urgent_stream.cuda_stream if self.urgent_stream is not None else None)
         self._h = C.c_void_p()
         self._keep = []
@@ -222,6 +223,10 @@ class Context:
     def select_topk(self, q, q_token, landmarks, n_pages, out_idx, out_scores=None, stream=None):
         self._check(lib.dd_select_topk(self._h, _ptr(q), q_token, _ptr(landmarks), _ptr(n_pages), _ptr(out_idx),
                                        _ptr(out_scores), _stream(stream)))
+
+    def select_topk_chunked(self, q, q_token, landmarks, n_pages, ctx_len, out_idx, out_scores=None, stream=None):
+        self._check(lib.dd_select_topk_chunked(self._h, _ptr(q), q_token, _ptr(landmarks), _ptr(n_pages), _ptr(ctx_len),
+                                               _ptr(out_idx), _ptr(out_scores), _stream(stream)))
 
     def gather_kv_from_host(self, host_kv_layer, idx, n_pages, slot, stream=None):
         self._check(lib.dd_gather_kv_from_host(self._h, _ptr(host_kv_layer), _ptr(idx), _ptr(n_pages), slot,

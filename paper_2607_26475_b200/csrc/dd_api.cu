@@ -59,6 +59,10 @@ static const char* dd_check_config(const dd_config* c) {
   if (c->select_mode != DD_SELECT_AUTO && c->select_mode != DD_SELECT_TWO_KERNELS) return "unknown select_mode";
   if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
   if (c->miss_correction != 0 && c->miss_correction != 1) return "miss_correction must be 0 or 1";
+  {
+    const int ct = c->landmark_chunk_tokens;
+    if (ct != 0 && ct != 16 && ct != 8 && ct != 4 && ct != 2 && ct != 1) return "landmark_chunk_tokens must be 0, 16, 8, 4, 2 or 1";
+  }
   if (c->attn_splits > 512) return "attn_splits must be <= 512";
   if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";
   if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
@@ -184,6 +188,7 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   }
   ctx->sm_count = dd_sm_count();
   ctx->G = cfg->n_q_heads / cfg->n_kv_heads;
+  ctx->R = cfg->landmark_chunk_tokens ? DD_T / cfg->landmark_chunk_tokens : 1;
   ctx->n_rows = cfg->n_q_tokens * ctx->G;
   ctx->score_tiles = (cfg->max_pages + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
   ctx->attn_splits = dd_resolve_splits(cfg, ctx->sm_count, &ctx->attn_cluster);
@@ -378,6 +383,21 @@ extern "C" int dd_select_topk(dd_ctx* ctx, const void* q, int q_token, const voi
                           (cudaStream_t)stream);
 }
 
+extern "C" int dd_select_topk_chunked(dd_ctx* ctx, const void* q, int q_token, const void* landmarks, const int* n_pages,
+                                      const int* ctx_len, int* out_idx, float* out_scores, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_select_topk_chunked: ctx is NULL");
+  if (q_token < 0 || q_token >= ctx->cfg.n_q_tokens)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "q_token %d outside [0, %d)", q_token, ctx->cfg.n_q_tokens);
+  DD_TRY(dd_check_dev(ctx, q, "q"));
+  DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
+  DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
+  DD_TRY(dd_check_dev(ctx, out_idx, "out_idx", 4));
+  if (out_scores) DD_TRY(dd_check_dev(ctx, out_scores, "out_scores", 4));
+  return dd_launch_select(ctx, q, q_token, ctx->cfg.n_q_tokens, landmarks, n_pages, out_idx, out_scores,
+                          (cudaStream_t)stream, ctx_len);
+}
+
 extern "C" int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, const int* idx, const int* n_pages,
                                       int slot, void* stream) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_gather_kv_from_host: ctx is NULL");
@@ -459,7 +479,7 @@ extern "C" int dd_prime(dd_ctx* ctx, const void* q_init) {
   const size_t q_layer = (size_t)c.batch * c.n_q_heads * DD_D;
   for (int l = 0; l < c.n_layers; ++l) {
     DD_TRY(dd_launch_select(ctx, (const __nv_bfloat16*)q_init + l * q_layer, 0, 1, ctx->landmarks[l], ctx->n_pages,
-                            dd_idx_of(ctx, 0, l), nullptr, cs));
+                            dd_idx_of(ctx, 0, l), nullptr, cs, ctx->ctx_len));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[l], cs));
   }
   for (int i = 0; i < DD_MAX_RING; ++i) ctx->released_recorded[i] = false;
@@ -494,7 +514,8 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
     // the next step runs on the compute stream while that transfer is in flight
     cudaStream_t us = (cudaStream_t)c.urgent_stream;
     int* merged = ctx->idx_merged + (size_t)slot * c.batch * c.n_kv_heads * c.k_pages;
-    DD_TRY(dd_launch_select(ctx, q, 0, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages, ctx->idx_true, nullptr, cs));
+    DD_TRY(dd_launch_select(ctx, q, 0, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages, ctx->idx_true, nullptr, cs,
+                            ctx->ctx_len));
     DD_TRY(dd_launch_diff(ctx, attn_idx, ctx->idx_true, slot, merged, cs));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->fix_ready[slot], cs));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->fix_ready[slot], 0));
@@ -502,7 +523,7 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
     DD_TRY(dd_launch_gather_fix(ctx, ctx->host_kv[layer], slot, us));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->urgent_done[slot], us));
     DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
-                            dd_idx_of(ctx, step + 1, layer), nullptr, cs));
+                            dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->urgent_done[slot], 0));            // all transfers of the layer complete
@@ -516,7 +537,7 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   ctx->released_recorded[slot] = true;
   if (!c.miss_correction) {
     DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
-                            dd_idx_of(ctx, step + 1, layer), nullptr, cs));
+                            dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
   }
   // the slot just released takes the gather `ahead` layers further on (index set known: it was

@@ -21,6 +21,7 @@ struct dd_ctx {
   int device;
   int sm_count;
   int G;                 // query heads per KV head
+  int R;                 // landmark chunks per page (1 = one landmark per page)
   int n_rows;            // Tq * G query rows that share one KV head
   int score_tiles;       // ceil(P / DD_SCORE_TILE)
   int attn_splits;       // resolved blocks per (request, KV head)
@@ -74,7 +75,7 @@ int dd_fail(dd_ctx* ctx, int code, const char* fmt, ...);
 // Launchers implemented next to their kernels; all asynchronous on `st`.
 int dd_launch_build_landmarks(dd_ctx* ctx, const void* kv_dev, const int* ctx_len, void* landmarks, cudaStream_t st);
 int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
-                     const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st);
+                     const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st, const int* ctx_len = nullptr);
 int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int* n_pages, char* slot, cudaStream_t st);
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
                    float* out_lse, cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr);

@@ -10,22 +10,25 @@
 #include "dd_common.cuh"
 
 // ------------------------------------------------------------------------------------------------
-// Landmarks: mean of the valid keys of a page, fp32 sum in token order, fp32 divide, RNE to bf16.
-// One warp per page; a lane owns 4 consecutive channels.
+// Landmarks: mean of the valid keys of a chunk (a page, or 1/R of a page), fp32 sum in token order, fp32
+// divide, RNE to bf16. One warp per chunk; a lane owns 4 consecutive channels.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) dd_landmark_kernel(const __nv_bfloat16* __restrict__ kv,
                                                           const int* __restrict__ ctx_len,
-                                                          __nv_bfloat16* __restrict__ lm, int Hkv, int P,
-                                                          long long n_pages_total) {
+                                                          __nv_bfloat16* __restrict__ lm, int Hkv, int P, int R,
+                                                          long long n_chunks_total) {
   const int lane = threadIdx.x & 31;
-  long long page = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int c = DD_T / R;                        // tokens per chunk
+  long long chunk = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long stride = (long long)gridDim.x * (blockDim.x >> 5);
-  for (; page < n_pages_total; page += stride) {
+  for (; chunk < n_chunks_total; chunk += stride) {
+    const long long page = chunk / R;
+    const int r = (int)(chunk - page * R);
     const int p = (int)(page % P);
     const int b = (int)(page / ((long long)P * Hkv));
-    int cnt = ctx_len[b] - p * DD_T;
-    cnt = cnt > DD_T ? DD_T : cnt;
-    const __nv_bfloat16* src = kv + page * (2 * DD_T * DD_D) + lane * 4;   // K half comes first
+    int cnt = ctx_len[b] - (p * DD_T + r * c);
+    cnt = cnt > c ? c : cnt;
+    const __nv_bfloat16* src = kv + page * (2 * DD_T * DD_D) + (size_t)r * c * DD_D + lane * 4;   // K half comes first
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
     for (int i = 0; i < cnt; ++i) {
       uint2 w = *reinterpret_cast<const uint2*>(src + i * DD_D);
@@ -38,25 +41,25 @@ __global__ void __launch_bounds__(256) dd_landmark_kernel(const __nv_bfloat16* _
     }
     uint2 o = make_uint2(0u, 0u);
     if (cnt > 0) {
-      const float c = (float)cnt;
-      __nv_bfloat162 lo = __floats2bfloat162_rn(__fdiv_rn(a0, c), __fdiv_rn(a1, c));
-      __nv_bfloat162 hi = __floats2bfloat162_rn(__fdiv_rn(a2, c), __fdiv_rn(a3, c));
+      const float n = (float)cnt;
+      __nv_bfloat162 lo = __floats2bfloat162_rn(__fdiv_rn(a0, n), __fdiv_rn(a1, n));
+      __nv_bfloat162 hi = __floats2bfloat162_rn(__fdiv_rn(a2, n), __fdiv_rn(a3, n));
       o.x = *reinterpret_cast<uint32_t*>(&lo);
       o.y = *reinterpret_cast<uint32_t*>(&hi);
     }
-    *reinterpret_cast<uint2*>(lm + page * DD_D + lane * 4) = o;
+    *reinterpret_cast<uint2*>(lm + chunk * DD_D + lane * 4) = o;
   }
 }
 
 int dd_launch_build_landmarks(dd_ctx* ctx, const void* kv_dev, const int* ctx_len, void* landmarks, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
-  const long long total = (long long)c.batch * c.n_kv_heads * c.max_pages;
+  const long long total = (long long)c.batch * c.n_kv_heads * c.max_pages * ctx->R;
   const int warps_per_block = 8;
   long long blocks = (total + warps_per_block - 1) / warps_per_block;
   const long long cap = (long long)ctx->sm_count * 16;
   if (blocks > cap) blocks = cap;
   dd_landmark_kernel<<<(unsigned)blocks, warps_per_block * 32, 0, st>>>(
-      (const __nv_bfloat16*)kv_dev, ctx_len, (__nv_bfloat16*)landmarks, c.n_kv_heads, c.max_pages, total);
+      (const __nv_bfloat16*)kv_dev, ctx_len, (__nv_bfloat16*)landmarks, c.n_kv_heads, c.max_pages, ctx->R, total);
   DD_CUDA_TRY(ctx, cudaGetLastError());
   return DD_OK;
 }
@@ -387,10 +390,11 @@ __device__ __forceinline__ unsigned dd_scan256_excl(unsigned v, unsigned* warp_t
 __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     const __nv_bfloat16* __restrict__ q, int q_req_stride, int q_token_off, const __nv_bfloat16* __restrict__ lm,
     const int* __restrict__ n_pages, int* __restrict__ out_idx, float* __restrict__ out_scores, int P, int G, int Hkv,
-    int k, int forced, int ppc, int* err_word) {
+    int k, int forced, int ppc, int* err_word, int R, const int* __restrict__ ctx_len) {
   extern __shared__ __align__(16) unsigned char sel_smem[];
-  float* s_sm = reinterpret_cast<float*>(sel_smem);                              // [ppc][G] logits; key in [p][0]
-  unsigned* hist = reinterpret_cast<unsigned*>(sel_smem + (size_t)ppc * G * 4);  // [2][RADIX_BINS]
+  float* s_sm = reinterpret_cast<float*>(sel_smem);                    // [ppc * R][G] logits; a page's key in its first slot
+  unsigned* hist = reinterpret_cast<unsigned*>(sel_smem + (size_t)ppc * R * G * 4);   // [2][RADIX_BINS]
+  const int KS = R * G;                                                // floats per page
   __shared__ float2 cta_ml[8];
   __shared__ unsigned cta_minmax[2];
   __shared__ unsigned cta_cnt[2];
@@ -421,6 +425,10 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   const int k_free = k_eff - forced_eff;
   const int p_lo = rank * ppc;
   const int n_local = max(0, min(np, p_lo + ppc) - p_lo);
+  // landmark rows (chunks) of this block: with R chunks per page only the chunks that hold a token exist
+  int n_rows_req = np * R;
+  if (R > 1) n_rows_req = min(n_rows_req, (ctx_len[b] + DD_T / R - 1) / (DD_T / R));
+  const int n_local_rows = max(0, min(n_rows_req, (p_lo + ppc) * R) - p_lo * R);
   if (tid == 0) { cta_minmax[0] = 0xFFFFFFFFu; cta_minmax[1] = 0u; cta_cnt[0] = 0u; cta_cnt[1] = 0u; cand_n = 0u; }
 
   DD_SEL_MARK(0);
@@ -438,14 +446,15 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) qf[kk] = make_uint4(0u, 0u, 0u, 0u);
     }
-    const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * DD_D;
+    const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * R * DD_D;
     const float scale = rsqrtf((float)DD_D);
-    for (int t0 = warp * 32; t0 < n_local; t0 += SEL_WARPS * 32) {     // two 16-page MMA tiles per trip
+    const int row_lo = p_lo * R, row_max = P * R - 1;
+    for (int t0 = warp * 32; t0 < n_local_rows; t0 += SEL_WARPS * 32) {  // two 16-row MMA tiles per trip
       uint4 lo[2][4], hi[2][4];
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const int pa = min(p_lo + t0 + mt * 16 + gl, P - 1);           // stay inside the tensor; discarded later
-        const int pb = min(p_lo + t0 + mt * 16 + gl + 8, P - 1);
+        const int pa = min(row_lo + t0 + mt * 16 + gl, row_max);       // stay inside the tensor; discarded later
+        const int pb = min(row_lo + t0 + mt * 16 + gl + 8, row_max);
         const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D);
         const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D);
 #pragma unroll
@@ -464,8 +473,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
         }
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          const int pl = t0 + mt * 16 + gl + r * 8;                     // page within the block
-          if (pl < n_local) {
+          const int pl = t0 + mt * 16 + gl + r * 8;                     // landmark row within the block
+          if (pl < n_local_rows) {
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
               const int h = 2 * t + c;
@@ -524,21 +533,25 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
     for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
       float c = -INFINITY;
+      for (int r = 0; r < R; ++r) {              // a page takes the best of its existing chunks
+        if (pl * R + r < n_local_rows) {
 #pragma unroll
-      for (int h = 0; h < 8; ++h)
-        if (h < G) c = fmaxf(c, s_sm[(size_t)pl * G + h] - lse[h]);
+          for (int h = 0; h < 8; ++h)
+            if (h < G) c = fmaxf(c, s_sm[((size_t)pl * R + r) * G + h] - lse[h]);
+        }
+      }
       const int p = p_lo + pl;
       if (out_scores) out_scores[bg * P + p] = expf(c);
       uint32_t key = dd_orderable(c);
       if (p >= n_free) key = 0xFFFFFFFFu;
       else { kmin = min(kmin, key); kmax = max(kmax, key); }
-      reinterpret_cast<uint32_t*>(s_sm)[(size_t)pl * G] = key;
+      reinterpret_cast<uint32_t*>(s_sm)[(size_t)pl * KS] = key;
     }
     kmin = __reduce_min_sync(0xffffffffu, kmin);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
     if (lane == 0) { atomicMin(&cta_minmax[0], kmin); atomicMax(&cta_minmax[1], kmax); }
   }
-  const uint32_t* keys = reinterpret_cast<const uint32_t*>(s_sm);      // key of local page pl at keys[pl * G]
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(s_sm);      // key of local page pl at keys[pl * KS]
   DD_SEL_MARK(3);
   cl.sync();
   DD_SEL_MARK(4);
@@ -570,7 +583,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) h[i] = 0u;
       __syncthreads();
       for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
-        const unsigned long long rel = (unsigned long long)(keys[(size_t)pl * G] - kmin);
+        const unsigned long long rel = (unsigned long long)(keys[(size_t)pl * KS] - kmin);
         if ((rel >> hi) == prefix) atomicAdd(&h[(unsigned)(rel >> shift) & ((1u << width) - 1u)], 1u);
       }
       __syncthreads();
@@ -612,7 +625,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       } else if (bin_cnt <= (unsigned)SEL_CAND_MAX) {
         // few keys share the prefix: every block lists its own, all blocks read all lists and rank them
         for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
-          const uint32_t key = keys[(size_t)pl * G];
+          const uint32_t key = keys[(size_t)pl * KS];
           if (((unsigned long long)(key - kmin) >> shift) == prefix) cand[atomicAdd(&cand_n, 1u)] = key;
         }
         cl.sync();
@@ -647,7 +660,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   {
     unsigned gt = 0, eq = 0;
     for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
-      const uint32_t key = keys[(size_t)pl * G];
+      const uint32_t key = keys[(size_t)pl * KS];
       if (p_lo + pl >= n_free || key > thr) ++gt;
       else if (key == thr) ++eq;
     }
@@ -667,7 +680,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     const int pl = c0 + tid;
     unsigned gt = 0, eq = 0;
     if (pl < n_local) {
-      const uint32_t key = keys[(size_t)pl * G];
+      const uint32_t key = keys[(size_t)pl * KS];
       if (p_lo + pl >= n_free || key > thr) gt = 1;
       else if (key == thr) eq = 1;
     }
@@ -688,9 +701,10 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
 }
 
 int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
-                     const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st) {
+                     const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st, const int* ctx_len) {
   const dd_config& c = ctx->cfg;
   const int G = ctx->G;
+  if (ctx->R > 1 && !ctx_len) return dd_fail(ctx, DD_ERR_INVALID_ARG, "finer landmarks need ctx_len for the selection");
   if (ctx->sel_cluster > 0) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->sel_cluster, c.n_kv_heads, c.batch);
@@ -707,7 +721,8 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
     DD_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, dd_select_fused_kernel, (const __nv_bfloat16*)q,
                                         q_tokens_in_tensor * c.n_q_heads * DD_D, q_token * c.n_q_heads * DD_D,
                                         (const __nv_bfloat16*)landmarks, n_pages, out_idx, out_scores, c.max_pages, G,
-                                        c.n_kv_heads, c.k_pages, c.forced_recent_pages, ctx->sel_ppc, ctx->err_word));
+                                        c.n_kv_heads, c.k_pages, c.forced_recent_pages, ctx->sel_ppc, ctx->err_word,
+                                        ctx->R, ctx_len));
     return DD_OK;
   }
   dim3 sgrid(ctx->score_tiles, c.n_kv_heads, c.batch);
@@ -743,7 +758,7 @@ static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
   for (; C <= c_max; C *= 2) {
     int ppc = (c.max_pages + C - 1) / C;
     ppc = (ppc + 31) & ~31;                                // whole pairs of MMA tiles
-    const size_t smem = (size_t)ppc * G * 4 + 2 * RADIX_BINS * 4;
+    const size_t smem = (size_t)ppc * ctx->R * G * 4 + 2 * RADIX_BINS * 4;
     if (smem > (size_t)SEL_MAX_SMEM) continue;             // too long for this cluster size: try a larger one
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(C, c.n_kv_heads, c.batch);
@@ -775,5 +790,8 @@ int dd_select_setup(dd_ctx* ctx) {
   ctx->sel_cluster = 0;
   if (ctx->cfg.select_mode != DD_SELECT_TWO_KERNELS)
     ctx->sel_cluster = dd_select_pick_cluster(ctx, &ctx->sel_ppc, &ctx->sel_smem_bytes);
+  if (ctx->R > 1 && ctx->sel_cluster == 0)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "finer landmarks are supported by the fused selection kernel only, and "
+                   "this request length does not fit it");
   return DD_OK;
 }

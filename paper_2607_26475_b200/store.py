@@ -45,7 +45,8 @@ class HostStore:
         for l in range(self.n_phys):
             host = torch.empty((B, w.n_kv_heads, w.n_pages, 2, w.page_tokens, w.head_dim), dtype=torch.bfloat16,
                                pin_memory=True)
-            lm = torch.empty((B, w.n_kv_heads, w.n_pages, w.head_dim), dtype=torch.bfloat16, device="cuda")
+            R = w.page_tokens // ctx.cfg.landmark_chunk_tokens if ctx.cfg.landmark_chunk_tokens else 1
+            lm = torch.empty((B, w.n_kv_heads, w.n_pages * R, w.head_dim), dtype=torch.bfloat16, device="cuda")
             for b in range(B):
                 slab = wl.kv_slab(w, l, b, device="cuda")
                 # landmarks of one request at a time: view the request as a batch of one
@@ -73,7 +74,8 @@ class HostStore:
             from . import binding
             c = ctx.cfg
             self._one = binding.Context(n_layers=1, batch=1, max_pages=c.max_pages, k_pages=1,
-                                        n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads)
+                                        n_q_heads=c.n_q_heads, n_kv_heads=c.n_kv_heads,
+                                        landmark_chunk_tokens=c.landmark_chunk_tokens)
         return self._one
 
     @property
