@@ -386,7 +386,7 @@ def main():
             "unit": "GB/s", "frac": gather_bytes / (gather_ms_live * 1e-3) / 1e9 / link_peak,
             "traffic": NCU_TRAFFIC["gather_dram"] * gather_bytes / (64 << 20),
             "link_traffic": NCU_TRAFFIC["gather_sysmem"] * gather_bytes / (64 << 20),
-            "traffic_source": "ncu capture of a 64 MiB launch (profiles/dd_gather_kernels_config2.md), scaled by gathered "
+            "traffic_source": "ncu capture of a 64 MiB launch (summary committed under profiles/), scaled by gathered "
                               "bytes: `traffic` = DRAM read+write (the slot stays in L2), `link_traffic` = sysmem sectors x 32 B",
             "peak_source": "pinned cudaMemcpyAsync host->device, 256 MiB, best of 6, measured in this run",
             "how": "gathered bytes per launch / (copy-stream span of the timed region / launches)",
