@@ -219,6 +219,12 @@ def main():
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        try:    # keep this replica's threads (and so its pinned store) on the CPUs next to its GPU
+            import pynvml
+            pynvml.nvmlInit()
+            pynvml.nvmlDeviceSetCpuAffinity(pynvml.nvmlDeviceGetHandleByIndex(local_rank))
+        except Exception as e:
+            log(f"rank {rank}: CPU affinity not set ({e})")
     w = wl.CONFIGS[args.config]
     if args.layers or args.batch:
         w = wl.small(w, n_layers=args.layers or w.n_layers, batch=args.batch or w.batch)
@@ -363,7 +369,8 @@ def main():
                 "d2h_bytes_per_step": o_bytes,
                 "note": "queries copied from pinned host memory and outputs read back every step, host waits for "
                         "each step; the KV gather from the host store is part of the path in both numbers"},
-        "gpu_launches": K * L * (7 if args.correct_misses else 3),
+        # per layer step: attention, selection, prefetch gather (+ true-index selection, diff, missing-page gather)
+        "gpu_launches": K * L * (6 if args.correct_misses else 3),
         "clocks": clocks,
     }
 
