@@ -61,6 +61,8 @@ def parse_args():
                          "step's current query (lower = more prediction misses)")
     ap.add_argument("--landmark-chunk", type=int, default=0,
                     help="tokens per landmark: 0/16 = one per page (default), 8/4/2/1 = several per page")
+    ap.add_argument("--no-select-stream", action="store_true",
+                    help="run the next-step selection on the compute stream instead of a stream of its own")
     ap.add_argument("--ragged", action="store_true", help="unequal context lengths per request (second workload shape)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-stages", action="store_true")
@@ -242,7 +244,8 @@ def main():
     ctx = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                      forced_recent_pages=w.forced_recent_pages, ring_depth=args.ring_depth, gather_mode=gm,
                      gather_ctas=args.gather_ctas, attn_splits=args.attn_splits, compute_stream=compute, copy_stream=copy,
-                     miss_correction=args.correct_misses, urgent_stream=urgent, landmark_chunk_tokens=args.landmark_chunk)
+                     miss_correction=args.correct_misses, urgent_stream=urgent, landmark_chunk_tokens=args.landmark_chunk,
+                     select_stream=None if args.no_select_stream else torch.cuda.Stream())
     budget = replicas.host_budget_per_rank(available_host_bytes(), world)
     store = HostStore(w, ctx, n_phys_layers=args.phys_layers or None, ragged=args.ragged, host_budget_bytes=budget,
                       log=log if rank == 0 else None)
@@ -358,7 +361,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "batch": B, "ctx": w.ctx, "budget": w.budget, "layers": L,
                    "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "landmark_chunk_tokens": args.landmark_chunk or w.page_tokens, "gather_mode": args.gather_mode,
+                   "page_tokens": w.page_tokens, "ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "select_stream": not args.no_select_stream, "landmark_chunk_tokens": args.landmark_chunk or w.page_tokens, "gather_mode": args.gather_mode,
                    "host_store_gib": store.host_bytes / 2**30, "phys_layers": store.n_phys,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2: each layer streams its own 32 MiB of landmarks and 64 MiB of "
@@ -478,13 +481,21 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n_rep = 4
+    ss = ctx.select_stream
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
     for r in range(n_rep + 1):
         if r == 1:
             e0.record(cs)
         for l in range(L):
-            ctx.sparse_decode_attn(q_dev[0, l], 0, idx[0], store.ctx_len_dev, outs[l], None, stream=cs)
+            if ss is not None:            # as in the pipelined step: selection next to the attention, joined afterwards
+                fork.record(cs)
+                ss.wait_event(fork)
             ctx.select_topk_chunked(q_dev[0, l], 1, store.landmarks[l], store.n_pages_dev, store.ctx_len_dev, tmp_idx,
-                                    None, stream=cs)
+                                    None, stream=ss if ss is not None else cs)
+            ctx.sparse_decode_attn(q_dev[0, l], 0, idx[0], store.ctx_len_dev, outs[l], None, stream=cs)
+            if ss is not None:
+                join.record(ss)
+                cs.wait_event(join)
     e1.record(cs)
     torch.cuda.synchronize()
     compute_only = e0.elapsed_time(e1) * 1e3 / (n_rep * L)

@@ -77,6 +77,8 @@ typedef struct dd_config {
   int landmark_chunk_tokens; /* tokens summarised by one landmark: 0 or 16 = one per page; 8, 4, 2, 1 = several per page */
   int miss_correction;       /* 1: dd_decode_layer_step repairs prediction misses before attention (needs urgent_stream) */
   void* urgent_stream;       /* cudaStream_t, ideally of higher priority than copy_stream; used for the missing pages */
+  void* select_stream;       /* optional cudaStream_t: the pipelined calls run the next-step selection there, concurrently
+                                with attention (the two are independent); NULL = on the compute stream */
 } dd_config;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -193,6 +195,8 @@ int dd_prime(dd_ctx* ctx, const void* q_init);
  *                   -> index set of (step+1, layer)
  *   copy stream:    wait released[slot] (and the selection it depends on) -> gather of layer
  *                   layer+D of this step, or of layer layer+D-L of the next step
+ * With a select_stream the selection runs there, next to the attention; the compute stream waits for it at the
+ * end of the call, so that work enqueued on the compute stream after this call may reuse q as before.
  *   q    dev bf16 [B][Tq][Hq][d]
  *   out  dev bf16 [B][Tq][Hq][d], written */
 int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out);

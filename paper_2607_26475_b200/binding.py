@@ -47,6 +47,7 @@ class DDConfig(C.Structure):
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
         ("landmark_chunk_tokens", C.c_int), ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
+        ("select_stream", C.c_void_p),
     ]
 
 
@@ -148,7 +149,7 @@ class Context:
     def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
                  gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None,
-                 miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0):
+                 miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0, select_stream=None):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
@@ -162,7 +163,9 @@ class Context:
                             self.compute_stream.cuda_stream, self.copy_stream.cuda_stream,
                             _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0,
                             landmark_chunk_tokens, 1 if miss_correction else 0,
-                            self.urgent_stream.cuda_stream if self.urgent_stream is not None else None)
+                            self.urgent_stream.cuda_stream if self.urgent_stream is not None else None,
+                            select_stream.cuda_stream if select_stream is not None else None)
+        self.select_stream = select_stream
         self._h = C.c_void_p()
         self._keep = []
         rc = lib.dd_create(C.byref(self.cfg), C.byref(self._h))

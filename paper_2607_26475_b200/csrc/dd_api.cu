@@ -160,6 +160,7 @@ static void dd_free_all(dd_ctx* ctx) {
     if (ctx->fix_ready[i]) cudaEventDestroy(ctx->fix_ready[i]);
     if (ctx->urgent_done[i]) cudaEventDestroy(ctx->urgent_done[i]);
   }
+  if (ctx->q_ready) cudaEventDestroy(ctx->q_ready);
   if (ctx->sel_done) {
     for (int l = 0; l < ctx->cfg.n_layers; ++l)
       if (ctx->sel_done[l]) cudaEventDestroy(ctx->sel_done[l]);
@@ -249,6 +250,7 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->fix_ready[i], cudaEventDisableTiming));
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->urgent_done[i], cudaEventDisableTiming));
   }
+  DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->q_ready, cudaEventDisableTiming));
   ctx->sel_done = new cudaEvent_t[cfg->n_layers]();
   for (int l = 0; l < cfg->n_layers; ++l)
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->sel_done[l], cudaEventDisableTiming));
@@ -270,9 +272,11 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
 extern "C" int dd_sync(dd_ctx* ctx, double timeout_s) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sync: ctx is NULL");
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(timeout_s);
-  cudaStream_t streams[3] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream,
-                             (cudaStream_t)ctx->cfg.urgent_stream};
-  for (int i = 0; i < (ctx->cfg.miss_correction ? 3 : 2); ++i) {
+  cudaStream_t streams[4] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream, nullptr, nullptr};
+  int n_streams = 2;
+  if (ctx->cfg.miss_correction) streams[n_streams++] = (cudaStream_t)ctx->cfg.urgent_stream;
+  if (ctx->cfg.select_stream) streams[n_streams++] = (cudaStream_t)ctx->cfg.select_stream;
+  for (int i = 0; i < n_streams; ++i) {
     for (;;) {
       cudaError_t e = cudaStreamQuery(streams[i]);
       if (e == cudaSuccess) break;
@@ -509,9 +513,22 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
 
   const int spec_token = c.n_q_tokens - 1;
   const int* attn_idx = dd_idx_of(ctx, step, layer);
+  // The selection of the next step's set is independent of this layer's attention. With a select stream it runs
+  // there (the two-kernel path shares scratch with the true-index selection, so under correction only the fused
+  // kernel may move); the compute stream rejoins it at the end of the call.
+  cudaStream_t ss = (cudaStream_t)c.select_stream;
+  const bool side_select = ss != nullptr && (!c.miss_correction || ctx->sel_cluster > 0);
+  cudaStream_t sel_st = side_select ? ss : cs;
+  if (side_select) {
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->q_ready, cs));
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(ss, ctx->q_ready, 0));
+    DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
+                            dd_idx_of(ctx, step + 1, layer), nullptr, sel_st, ctx->ctx_len));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], sel_st));
+  }
   if (c.miss_correction) {
     // true index from the current token, repair list, missing pages on the urgent stream; the selection for
-    // the next step runs on the compute stream while that transfer is in flight
+    // the next step runs while that transfer is in flight
     cudaStream_t us = (cudaStream_t)c.urgent_stream;
     int* merged = ctx->idx_merged + (size_t)slot * c.batch * c.n_kv_heads * c.k_pages;
     DD_TRY(dd_launch_select(ctx, q, 0, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages, ctx->idx_true, nullptr, cs,
@@ -522,9 +539,11 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->ready[slot], 0));                  // the prefetch wrote the slot first
     DD_TRY(dd_launch_gather_fix(ctx, ctx->host_kv[layer], slot, us));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->urgent_done[slot], us));
-    DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
-                            dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
-    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+    if (!side_select) {
+      DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
+                              dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
+      DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+    }
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->urgent_done[slot], 0));            // all transfers of the layer complete
     attn_idx = merged;
@@ -535,11 +554,12 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
                         k_new, v_new));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
   ctx->released_recorded[slot] = true;
-  if (!c.miss_correction) {
+  if (!c.miss_correction && !side_select) {
     DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
                             dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
   }
+  if (side_select) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->sel_done[layer], 0));   // q may be reused after this call
   // the slot just released takes the gather `ahead` layers further on (index set known: it was
   // selected one step earlier, or just now when the ring is deeper than the model)
   const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;

@@ -53,6 +53,7 @@ struct dd_ctx {
   cudaEvent_t released[DD_MAX_RING];
   bool released_recorded[DD_MAX_RING];
   cudaEvent_t* sel_done;  // [L]
+  cudaEvent_t q_ready;    // start of a layer step on the compute stream (the select stream starts from it)
   cudaEvent_t fix_ready[DD_MAX_RING];    // fix list of the slot written (compute stream)
   cudaEvent_t urgent_done[DD_MAX_RING];  // missing pages of the slot fetched (urgent stream)
   // bound tables

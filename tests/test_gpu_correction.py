@@ -64,11 +64,12 @@ def _inputs(w, S):
     return store, lms, ctx_len, npg, q_init, q_steps
 
 
-def _run(dd, w, S, inp, depth, correct, read=True):
+def _run(dd, w, S, inp, depth, correct, read=True, side_select=False):
     store, lms, ctx_len, npg, q_init, q_steps = inp
     L, B = w.n_layers, w.batch
     c = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
-                   forced_recent_pages=w.forced_recent_pages, ring_depth=depth, miss_correction=correct)
+                   forced_recent_pages=w.forced_recent_pages, ring_depth=depth, miss_correction=correct,
+                   select_stream=torch.cuda.Stream() if side_select else None)
     c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
     c.prime(q_init.cuda())
     qd = q_steps.cuda()
@@ -119,6 +120,9 @@ def test_corrected_chain_attends_the_true_sets(dd):
         o2, m2, _ = _run(dd, w, S, inp2, depth=depth, correct=True)
         assert np.array_equal(np.sort(m2, axis=-1), np.sort(merged, axis=-1))
         assert np.abs(f32(o2) - f32(outs)).max() <= 2e-2
+    # the next-step selection on its own stream changes nothing
+    o4, m4, _ = _run(dd, w, S, inp, depth=2, correct=True, side_select=True)
+    assert np.array_equal(m4, merged) and np.array_equal(raw16(o4), raw16(outs))
     # without correction the outputs are those of the predicted sets: they differ
     o3, _, _ = _run(dd, w, S, inp, depth=2, correct=False)
     assert np.abs(f32(o3) - f32(outs)).max() > 1e-3

@@ -32,13 +32,15 @@ def _inputs(w, S, ragged=True):
     return store, lms, ctx_len, npg, q_init, q_steps
 
 
-def _run(dd, w, S, inp, depth, mode=0, read_idx=True, one_stream=False):
+def _run(dd, w, S, inp, depth, mode=0, read_idx=True, one_stream=False, side_select=False):
     store, lms, ctx_len, npg, q_init, q_steps = inp
     L, B = w.n_layers, w.batch
     streams = {}
     if one_stream:                # fully synchronous schedule: gathers, attention and selection on one stream
         st = torch.cuda.Stream()
         streams = dict(compute_stream=st, copy_stream=st)
+    if side_select:               # the next-step selection on a stream of its own, next to the attention
+        streams = dict(select_stream=torch.cuda.Stream())
     c = dd.Context(n_layers=L, batch=B, max_pages=w.n_pages, k_pages=w.k_pages,
                    forced_recent_pages=w.forced_recent_pages, ring_depth=depth, gather_mode=mode, **streams)
     lm_dev = [x.cuda() for x in lms]
@@ -84,8 +86,9 @@ def test_chain_matches_oracle_and_is_invariant_to_ring_depth_and_engine(dd):
     # same bits whatever the ring depth, the gather engine, with no host reads in between, and with the whole
     # schedule serialised on a single stream
     for depth, mode, read, one in [(3, 0, True, False), (4, 0, False, False), (2, 1, False, False), (2, 0, False, False),
-                                   (2, 0, False, True)]:
-        o2, i2 = _run(dd, w, S, inp, depth=depth, mode=mode, read_idx=read, one_stream=one)
+                                   (2, 0, False, True), (2, 0, False, "side")]:
+        o2, i2 = _run(dd, w, S, inp, depth=depth, mode=mode, read_idx=read, one_stream=one is True,
+                      side_select=one == "side")
         assert np.array_equal(raw16(o2), raw16(outs)), (depth, mode, one)
         if read:
             assert np.array_equal(i2, idxs)
