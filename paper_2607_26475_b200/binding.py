@@ -58,9 +58,13 @@ class DDError(RuntimeError):
 
 
 def _load() -> C.CDLL:
-    if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_26475_b200.build` "
-                          "(there is no CPU fallback)")
+    from . import build as _build
+    try:
+        _build.build()          # compiles with nvcc when the library is missing or older than its sources
+    except Exception as e:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing and could not be built ({e}); build it with "
+                              "`python -m paper_2607_26475_b200.build` (there is no CPU fallback)") from e
     lib = C.CDLL(LIB_PATH)
     vp, ip = C.c_void_p, C.c_int
     lib.dd_create.argtypes = [C.POINTER(DDConfig), C.POINTER(vp)]
