@@ -477,6 +477,9 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     attn = lambda i: ctx.sparse_decode_attn(q_dev[0, 0], 0, idx[0], store.ctx_len_dev, outs[0], None, stream=cs)
     att_warm = timed(cs, attn)
     att_cold = timed(cs, attn, pre=flush_l2)
+    # load-only twins: what the memory system delivers for the same launch shape and size without any arithmetic
+    att_loads = timed(cs, lambda i: ctx.probe_attn_loads(0, stream=cs), pre=flush_l2)
+    sel_loads = timed(cs, lambda i: ctx.probe_select_loads(store.landmarks[i % L], store.n_pages_dev, stream=cs))
     # compute-only step: attention + selection of every layer with the slot already filled
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -504,15 +507,18 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     gb = w.gathered_bytes_per_layer
     return {
         "select_us": sel_us, "gather_us": gat_us, "attn_us_l2_warm": att_warm, "attn_us_l2_flushed": att_cold,
+        "select_loads_only_us": sel_loads, "attn_loads_only_us_l2_flushed": att_loads,
         "compute_only_us_per_layer": compute_only, "reps": reps,
         "roofline_kernels": {
             "dd_select_fused_kernel": {"bound": "hbm", "achieved": sel_bytes / (sel_us * 1e-6) / 1e9,
                                        "peak": hbm_peak, "unit": "GB/s",
                                        "frac": sel_bytes / (sel_us * 1e-6) / 1e9 / hbm_peak,
-                                       "traffic": NCU_TRAFFIC["select_dram"] * lm_bytes / (32 << 20)},
+                                       "traffic": NCU_TRAFFIC["select_dram"] * lm_bytes / (32 << 20),
+                                       "frac_of_load_only_kernel": sel_loads / sel_us},
             "dd_attn_kernel(l2 flushed)": {"bound": "hbm", "achieved": gb / (att_cold * 1e-6) / 1e9, "peak": hbm_peak,
                                            "unit": "GB/s", "frac": gb / (att_cold * 1e-6) / 1e9 / hbm_peak,
-                                           "traffic": NCU_TRAFFIC["attn_dram"] * gb / (64 << 20)},
+                                           "traffic": NCU_TRAFFIC["attn_dram"] * gb / (64 << 20),
+                                           "frac_of_load_only_kernel": att_loads / att_cold},
             "gather(alone)": {"bound": "host_link", "achieved": gb / (gat_us * 1e-6) / 1e9, "peak": link_peak,
                               "unit": "GB/s", "frac": gb / (gat_us * 1e-6) / 1e9 / link_peak},
         },

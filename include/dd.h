@@ -239,6 +239,17 @@ int dd_get_merged_indices(dd_ctx* ctx, int slot, const int** dev_idx);
 /* Synchronises, then reports how many pages were missing and how many were selected since the last reset. */
 int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset);
 
+/* ---- measurement aids ------------------------------------------------------------------------------- */
+
+/* Load-only twins of the two HBM-bound kernels: the same grid, the same walk over pages / landmark rows and the
+ * same 16-byte fragment loads as dd_sparse_decode_attn (over ring slot `slot`) and as the fused selection
+ * (over `landmarks`, dev bf16 [B][Hkv][P*R][d], with n_pages dev int32 [B]), but no arithmetic, no exchange and
+ * no output. Their duration is what the memory system delivers for that launch shape and size; the benchmark
+ * reports it next to the kernels' own times. dd_probe_select_loads needs the fused selection path
+ * (DD_ERR_STATE otherwise). Asynchronous on `stream`. */
+int dd_probe_attn_loads(dd_ctx* ctx, int slot, void* stream);
+int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const int* n_pages, void* stream);
+
 /* ---- attention without any allocation ----------------------------------------------------------- */
 
 /* (The paper has no counterpart of this call; it exists for integration.)

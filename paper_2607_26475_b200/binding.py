@@ -33,7 +33,7 @@ EXPORTS = [
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
-    "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats",
+    "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
 ]
 
 
@@ -94,6 +94,8 @@ def _load() -> C.CDLL:
     lib.dd_fetch_missing_from_host.argtypes = [vp, vp, ip, vp]
     lib.dd_get_merged_indices.argtypes = [vp, ip, C.POINTER(vp)]
     lib.dd_miss_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong), ip]
+    lib.dd_probe_attn_loads.argtypes = [vp, ip, vp]
+    lib.dd_probe_select_loads.argtypes = [vp, vp, vp, vp]
     lib.dd_static_scratch_capacity.argtypes = []
     lib.dd_static_scratch_capacity.restype = C.c_size_t
     lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7
@@ -283,6 +285,12 @@ class Context:
         a, b = C.c_ulonglong(), C.c_ulonglong()
         self._check(lib.dd_miss_stats(self._h, C.byref(a), C.byref(b), 1 if reset else 0))
         return a.value, b.value
+
+    def probe_attn_loads(self, slot, stream=None):
+        self._check(lib.dd_probe_attn_loads(self._h, slot, _stream(stream)))
+
+    def probe_select_loads(self, landmarks, n_pages, stream=None):
+        self._check(lib.dd_probe_select_loads(self._h, _ptr(landmarks), _ptr(n_pages), _stream(stream)))
 
     def get_indices(self, step_parity, layer) -> torch.Tensor:
         """A copy of the index set [B, Hkv, k] int32 used at (step parity, layer) (synchronises)."""

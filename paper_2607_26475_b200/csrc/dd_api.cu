@@ -118,7 +118,7 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
   z.topk_keys = up256(B * Hkv * P * 4);
   z.part_o = up256(B * Hkv * (size_t)S * 8 * DD_D * 4);
   z.part_ml = up256(B * Hkv * (size_t)S * 8 * 8);
-  z.ticket = up256(B * Hkv * 4);
+  z.ticket = up256(B * Hkv * 4 + 4);               // arrival counters + one word the load-only probes may write
   z.idx_tab = up256((size_t)2 * c->n_layers * B * Hkv * c->k_pages * 4);
   z.err = 256;
   const size_t sel = B * Hkv * (size_t)c->k_pages, D = c->ring_depth;
@@ -640,4 +640,18 @@ extern "C" int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned 
   if (missing) *missing = w[0];
   if (selected) *selected = w[1];
   return DD_OK;
+}
+
+extern "C" int dd_probe_attn_loads(dd_ctx* ctx, int slot, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_probe_attn_loads: ctx is NULL");
+  if (slot < 0 || slot >= ctx->cfg.ring_depth)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "slot %d outside [0, %d)", slot, ctx->cfg.ring_depth);
+  return dd_launch_attn_loads_only(ctx, ctx->ring + (size_t)slot * ctx->slot_bytes, (cudaStream_t)stream);
+}
+
+extern "C" int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const int* n_pages, void* stream) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_probe_select_loads: ctx is NULL");
+  DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
+  DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
+  return dd_launch_select_loads_only(ctx, landmarks, n_pages, (cudaStream_t)stream);
 }

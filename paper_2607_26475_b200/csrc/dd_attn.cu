@@ -438,6 +438,44 @@ int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx,
 }
 
 // ------------------------------------------------------------------------------------------------
+// Measurement aid: the attention kernel's loads and nothing else (same grid, same page walk, same fragment
+// addresses, no arithmetic, no merge). Its duration is what the memory system delivers for this launch shape.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_loads_only_kernel(const char* __restrict__ slot, int Hkv, int k,
+                                                                             int pages_per_split,
+                                                                             unsigned int* __restrict__ sink) {
+  const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const size_t bg = (size_t)b * Hkv + g;
+  const char* kbase = slot + bg * 2 * (size_t)k * DD_HALF_PAGE_BYTES;
+  const char* vbase = kbase + (size_t)k * DD_HALF_PAGE_BYTES;
+  const int p_begin = split * pages_per_split;
+  const int p_end = min(k, p_begin + pages_per_split);
+  unsigned int acc = 0;
+  for (int j = p_begin + warp; j < p_end; j += ATTN_WARPS) {
+    uint4 klo[4], khi[4], v[4][2];
+    dd_load_k(kbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, klo, khi);
+    dd_load_v(vbase + (size_t)j * DD_HALF_PAGE_BYTES, gl, t, v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc ^= klo[i].x ^ klo[i].y ^ klo[i].z ^ klo[i].w ^ khi[i].x ^ khi[i].y ^ khi[i].z ^ khi[i].w;
+      acc ^= v[i][0].x ^ v[i][0].y ^ v[i][0].z ^ v[i][0].w ^ v[i][1].x ^ v[i][1].y ^ v[i][1].z ^ v[i][1].w;
+    }
+  }
+  if (acc == 0x9E3779B9u) sink[0] = acc;        // keeps the loads alive; practically never true
+}
+
+int dd_launch_attn_loads_only(dd_ctx* ctx, const char* slot, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const int S = ctx->attn_splits;
+  dd_attn_loads_only_kernel<<<dim3(S, c.n_kv_heads, c.batch), ATTN_THREADS, 0, st>>>(
+      slot, c.n_kv_heads, c.k_pages, (c.k_pages + S - 1) / S, ctx->attn_ticket + c.batch * c.n_kv_heads);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
 // Allocation-free variant of the attention entry point.
 //
 // Some callers must not allocate device memory: code running between other libraries' memory pools,

@@ -700,6 +700,55 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   DD_SEL_MARK(7);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Measurement aid: the fused selection kernel's landmark loads and nothing else (same grid and block shape,
+// same rows per block, same fragment addresses; no arithmetic, no exchange).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_loads_only_kernel(const __nv_bfloat16* __restrict__ lm,
+                                                                              const int* __restrict__ n_pages, int P,
+                                                                              int Hkv, int ppc, int R,
+                                                                              unsigned int* __restrict__ sink) {
+  const int rank = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const size_t bg = (size_t)b * Hkv + g;
+  const int np = min(n_pages[b], P);
+  const int row_lo = rank * ppc * R, row_max = P * R - 1;
+  const int n_local_rows = max(0, min(np * R, row_lo + ppc * R) - row_lo);
+  const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * R * DD_D;
+  unsigned int acc = 0;
+  for (int t0 = warp * 32; t0 < n_local_rows; t0 += SEL_WARPS * 32) {
+    uint4 lo[2][4], hi[2][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+      const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)min(row_lo + t0 + mt * 16 + gl, row_max) * DD_D);
+      const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)min(row_lo + t0 + mt * 16 + gl + 8, row_max) * DD_D);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        lo[mt][kk] = dd_ld_stream(ra + kk * 4 + t);
+        hi[mt][kk] = dd_ld_stream(rb + kk * 4 + t);
+      }
+    }
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk)
+        acc ^= lo[mt][kk].x ^ lo[mt][kk].y ^ lo[mt][kk].z ^ lo[mt][kk].w ^ hi[mt][kk].x ^ hi[mt][kk].y ^ hi[mt][kk].z ^
+               hi[mt][kk].w;
+  }
+  if (acc == 0x9E3779B9u) sink[0] = acc;        // keeps the loads alive; practically never true
+}
+
+int dd_launch_select_loads_only(dd_ctx* ctx, const void* landmarks, const int* n_pages, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  if (ctx->sel_cluster <= 0) return dd_fail(ctx, DD_ERR_STATE, "the load-only probe follows the fused selection kernel");
+  dd_select_loads_only_kernel<<<dim3(ctx->sel_cluster, c.n_kv_heads, c.batch), SEL_THREADS, 0, st>>>(
+      (const __nv_bfloat16*)landmarks, n_pages, c.max_pages, c.n_kv_heads, ctx->sel_ppc, ctx->R,
+      ctx->attn_ticket + c.batch * c.n_kv_heads);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}
+
 int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
                      const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st, const int* ctx_len) {
   const dd_config& c = ctx->cfg;
