@@ -324,6 +324,29 @@ def main():
     gather_bytes = w.gathered_bytes_per_layer
     gather_ms_live = copy_ms / n_gathers
 
+    # ---- traced pass (outside the timed region): where the compute stream waits, how long the live gathers take
+    trace_steps = min(K, 4)
+    ctx.sync()
+    ctx.prime(q_init)
+    run_steps(0, W, 0)
+    ctx.trace_begin(trace_steps * L)
+    run_steps(W, W + trace_steps, W)
+    tr = ctx.trace_end()
+    pipeline_trace = None
+    if len(tr) > 2 * L:
+        import numpy as np
+        t = tr[L:]                                   # drop the first traced step (pipeline refill after the sync)
+        stall, attn_t, step_t, gath = t[:, 1] - t[:, 0], t[:, 2] - t[:, 1], t[:, 3] - t[:, 0], t[:, 5] - t[:, 4]
+        period = np.diff(t[:, 2])                    # attention-done to attention-done = layer period
+        pipeline_trace = {
+            "layer_steps": int(len(t)),
+            "compute_stall_on_transfer_us": {"median": float(np.median(stall)), "p90": float(np.percentile(stall, 90))},
+            "attention_us": float(np.median(attn_t)),
+            "gather_us_live": {"median": float(np.median(gath)), "p90": float(np.percentile(gath, 90))},
+            "layer_period_us": float(np.median(period)),
+            "exposed_transfer_fraction_of_period": float(np.median(stall) / np.median(period)),
+        }
+
     # ---- end-to-end run: every step copies its queries from pinned host memory, reads the outputs back
     ctx.sync()
     ctx.prime(q_init)
@@ -375,6 +398,7 @@ def main():
         # per layer step: attention, selection, prefetch gather (+ true-index selection, diff, missing-page gather)
         "gpu_launches": K * L * (6 if args.correct_misses else 3),
         "clocks": clocks,
+        "pipeline_trace": pipeline_trace,
     }
 
     if miss is not None:

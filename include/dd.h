@@ -239,6 +239,24 @@ int dd_get_merged_indices(dd_ctx* ctx, int slot, const int** dev_idx);
 /* Synchronises, then reports how many pages were missing and how many were selected since the last reset. */
 int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset);
 
+/* ---- timeline of the pipelined calls ------------------------------------------------------------------ */
+
+/* dd_trace_begin arms a timeline of up to max_layer_steps calls of dd_decode_layer_step (it creates timing
+ * events; no device memory). Every traced call records six points, in microseconds since the first traced call:
+ *   [0] the compute stream reaches the layer step (all earlier compute work done)
+ *   [1] every transfer the layer needs is complete: attention starts ([1] - [0] = time the compute stream
+ *       was stalled on the host link, plus the true-index selection and diff under miss correction)
+ *   [2] attention done (buffer released)
+ *   [3] end of the layer step on the compute stream (selection done or rejoined)
+ *   [4] the gather this call enqueued (layer + ring depth) starts on the copy stream, its waits satisfied
+ *   [5] that gather is complete
+ * dd_trace_end stops recording, synchronises and returns the number of traced calls; dd_trace_read copies
+ * `count` rows of 6 floats starting at row `first` into host memory `out`. DD_ERR_STATE when no trace exists. */
+#define DD_TRACE_FIELDS 6
+int dd_trace_begin(dd_ctx* ctx, int max_layer_steps);
+int dd_trace_end(dd_ctx* ctx, int* n_recorded);
+int dd_trace_read(dd_ctx* ctx, int first, int count, float* out);
+
 /* ---- measurement aids ------------------------------------------------------------------------------- */
 
 /* Load-only twins of the two HBM-bound kernels: the same grid, the same walk over pages / landmark rows and the

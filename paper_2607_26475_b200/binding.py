@@ -33,7 +33,9 @@ EXPORTS = [
     "dd_strerror", "dd_last_error_message", "dd_device_error", "dd_sync", "dd_build_landmarks",
     "dd_select_topk", "dd_gather_kv_from_host", "dd_sparse_decode_attn", "dd_bind", "dd_prime",
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
-    "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices", "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
+    "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices",
+    "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
+    "dd_trace_begin", "dd_trace_end", "dd_trace_read",
 ]
 
 
@@ -94,6 +96,9 @@ def _load() -> C.CDLL:
     lib.dd_fetch_missing_from_host.argtypes = [vp, vp, ip, vp]
     lib.dd_get_merged_indices.argtypes = [vp, ip, C.POINTER(vp)]
     lib.dd_miss_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong), ip]
+    lib.dd_trace_begin.argtypes = [vp, ip]
+    lib.dd_trace_end.argtypes = [vp, C.POINTER(ip)]
+    lib.dd_trace_read.argtypes = [vp, ip, ip, vp]
     lib.dd_probe_attn_loads.argtypes = [vp, ip, vp]
     lib.dd_probe_select_loads.argtypes = [vp, vp, vp, vp]
     lib.dd_static_scratch_capacity.argtypes = []
@@ -285,6 +290,19 @@ class Context:
         a, b = C.c_ulonglong(), C.c_ulonglong()
         self._check(lib.dd_miss_stats(self._h, C.byref(a), C.byref(b), 1 if reset else 0))
         return a.value, b.value
+
+    def trace_begin(self, max_layer_steps: int):
+        self._check(lib.dd_trace_begin(self._h, max_layer_steps))
+
+    def trace_end(self):
+        """Stops the trace and returns it as a [n, 6] float32 numpy array of microseconds (see dd_trace_begin)."""
+        import numpy as np
+        n = C.c_int()
+        self._check(lib.dd_trace_end(self._h, C.byref(n)))
+        out = np.zeros((n.value, 6), dtype=np.float32)
+        if n.value:
+            self._check(lib.dd_trace_read(self._h, 0, n.value, out.ctypes.data_as(C.c_void_p)))
+        return out
 
     def probe_attn_loads(self, slot, stream=None):
         self._check(lib.dd_probe_attn_loads(self._h, slot, _stream(stream)))

@@ -166,6 +166,12 @@ static void dd_free_all(dd_ctx* ctx) {
       if (ctx->sel_done[l]) cudaEventDestroy(ctx->sel_done[l]);
     delete[] ctx->sel_done;
   }
+  if (ctx->trace_ev) {
+    for (int i = 0; i < ctx->trace_cap * DD_TRACE_FIELDS; ++i)
+      if (ctx->trace_ev[i]) cudaEventDestroy(ctx->trace_ev[i]);
+    delete[] ctx->trace_ev;
+  }
+  if (ctx->trace_origin) cudaEventDestroy(ctx->trace_origin);
   delete[] ctx->landmarks;
   delete[] ctx->host_kv;
   delete ctx;
@@ -459,15 +465,17 @@ static int* dd_idx_of(dd_ctx* ctx, int parity, int layer) {
 
 // Gather number n = step * L + layer goes to slot n % D. It may start once the attention that last
 // read the slot has released it and the selection that produced its index set is done.
-static int dd_enqueue_gather(dd_ctx* ctx, long long n) {
+static int dd_enqueue_gather(dd_ctx* ctx, long long n, cudaEvent_t ev_start = nullptr, cudaEvent_t ev_end = nullptr) {
   const dd_config& c = ctx->cfg;
   const int layer = (int)(n % c.n_layers), step = (int)(n / c.n_layers);
   const int slot = (int)(n % c.ring_depth);
   cudaStream_t xs = (cudaStream_t)c.copy_stream;
   if (ctx->released_recorded[slot]) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->released[slot], 0));
   DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->sel_done[layer], 0));
+  if (ev_start) DD_CUDA_TRY(ctx, cudaEventRecord(ev_start, xs));
   DD_TRY(dd_launch_gather(ctx, ctx->host_kv[layer], dd_idx_of(ctx, step, layer), ctx->n_pages,
                           ctx->ring + (size_t)slot * ctx->slot_bytes, xs));
+  if (ev_end) DD_CUDA_TRY(ctx, cudaEventRecord(ev_end, xs));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->ready[slot], xs));
   return DD_OK;
 }
@@ -510,6 +518,13 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   if (k_new) DD_TRY(dd_check_dev(ctx, v_new, "v_new"));
   cudaStream_t cs = (cudaStream_t)c.compute_stream;
   const int slot = (int)(n % c.ring_depth);
+  cudaEvent_t* tr = nullptr;                     // this call's six timeline events, when a trace is armed
+  if (ctx->trace_on && ctx->trace_n < ctx->trace_cap) {
+    tr = ctx->trace_ev + (size_t)ctx->trace_n * DD_TRACE_FIELDS;
+    if (ctx->trace_n == 0) DD_CUDA_TRY(ctx, cudaEventRecord(ctx->trace_origin, cs));
+    DD_CUDA_TRY(ctx, cudaEventRecord(tr[0], cs));
+    ++ctx->trace_n;
+  }
 
   const int spec_token = c.n_q_tokens - 1;
   const int* attn_idx = dd_idx_of(ctx, step, layer);
@@ -550,8 +565,10 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   } else {
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));                  // transfer complete
   }
+  if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[1], cs));
   DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, attn_idx, ctx->ctx_len, out, nullptr, cs,
                         k_new, v_new));
+  if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[2], cs));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
   ctx->released_recorded[slot] = true;
   if (!c.miss_correction && !side_select) {
@@ -562,8 +579,9 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   if (side_select) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->sel_done[layer], 0));   // q may be reused after this call
   // the slot just released takes the gather `ahead` layers further on (index set known: it was
   // selected one step earlier, or just now when the ring is deeper than the model)
+  if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[3], cs));
   const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
-  DD_TRY(dd_enqueue_gather(ctx, n + ahead));
+  DD_TRY(dd_enqueue_gather(ctx, n + ahead, tr ? tr[4] : nullptr, tr ? tr[5] : nullptr));
   ctx->next_call = n + 1;
   return DD_OK;
 }
@@ -654,4 +672,47 @@ extern "C" int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const i
   DD_TRY(dd_check_dev(ctx, landmarks, "landmarks"));
   DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
   return dd_launch_select_loads_only(ctx, landmarks, n_pages, (cudaStream_t)stream);
+}
+
+extern "C" int dd_trace_begin(dd_ctx* ctx, int max_layer_steps) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_trace_begin: ctx is NULL");
+  if (max_layer_steps < 1 || max_layer_steps > (1 << 20)) return dd_fail(ctx, DD_ERR_INVALID_ARG, "max_layer_steps out of range");
+  DD_TRY(dd_sync(ctx, 60.0));
+  if (ctx->trace_ev) {
+    for (int i = 0; i < ctx->trace_cap * DD_TRACE_FIELDS; ++i)
+      if (ctx->trace_ev[i]) cudaEventDestroy(ctx->trace_ev[i]);
+    delete[] ctx->trace_ev;
+    ctx->trace_ev = nullptr;
+  }
+  if (!ctx->trace_origin) DD_CUDA_TRY(ctx, cudaEventCreate(&ctx->trace_origin));
+  ctx->trace_cap = max_layer_steps;
+  ctx->trace_n = 0;
+  ctx->trace_ev = new cudaEvent_t[(size_t)max_layer_steps * DD_TRACE_FIELDS]();
+  for (int i = 0; i < max_layer_steps * DD_TRACE_FIELDS; ++i) DD_CUDA_TRY(ctx, cudaEventCreate(&ctx->trace_ev[i]));
+  ctx->trace_on = true;
+  return DD_OK;
+}
+
+extern "C" int dd_trace_end(dd_ctx* ctx, int* n_recorded) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_trace_end: ctx is NULL");
+  if (!ctx->trace_ev) return dd_fail(ctx, DD_ERR_STATE, "dd_trace_end: no trace was begun");
+  ctx->trace_on = false;
+  DD_TRY(dd_sync(ctx, 120.0));
+  if (n_recorded) *n_recorded = ctx->trace_n;
+  return DD_OK;
+}
+
+extern "C" int dd_trace_read(dd_ctx* ctx, int first, int count, float* out) {
+  if (!ctx || !out) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_trace_read: NULL argument");
+  if (!ctx->trace_ev || ctx->trace_on) return dd_fail(ctx, DD_ERR_STATE, "dd_trace_read: end the trace first");
+  if (first < 0 || count < 0 || first + count > ctx->trace_n)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "rows [%d, %d) outside the %d traced calls", first, first + count, ctx->trace_n);
+  for (int i = 0; i < count; ++i) {
+    for (int f = 0; f < DD_TRACE_FIELDS; ++f) {
+      float ms = 0.f;
+      DD_CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->trace_origin, ctx->trace_ev[(size_t)(first + i) * DD_TRACE_FIELDS + f]));
+      out[(size_t)i * DD_TRACE_FIELDS + f] = ms * 1e3f;
+    }
+  }
+  return DD_OK;
 }

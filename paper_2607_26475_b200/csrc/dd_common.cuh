@@ -63,6 +63,11 @@ struct dd_ctx {
   const int* ctx_len;
   bool bound, primed;
   long long next_call;     // step * L + layer expected by dd_decode_layer_step
+  // optional timeline of the pipelined calls: DD_TRACE_FIELDS timing events per layer step
+  cudaEvent_t* trace_ev;
+  cudaEvent_t trace_origin;
+  int trace_cap, trace_n;
+  bool trace_on;
   char errmsg[512];
 };
 

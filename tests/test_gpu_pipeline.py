@@ -141,6 +141,37 @@ def test_layer_step_with_causal_tail(dd):
     c.close()
 
 
+def test_timeline_of_the_layer_steps(dd):
+    """Six timing points per layer step: monotone on the compute stream, gathers with positive duration, and the
+    gather a call enqueues finishes before the attention that consumes its slot starts."""
+    S = 3
+    w = wl.small(wl.CONFIGS[2], n_layers=4, batch=2, ctx=16 * 200, budget=16 * 40)
+    store, lms, ctx_len, npg, q_init, q_steps = _inputs(w, S)
+    L, depth = w.n_layers, 2
+    c = dd.Context(n_layers=L, batch=w.batch, max_pages=w.n_pages, k_pages=w.k_pages, ring_depth=depth)
+    with pytest.raises(dd.DDError) as e:
+        c.trace_end()
+    assert e.value.code == dd.DD_ERR_STATE
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qd = q_steps.cuda()
+    outs = torch.zeros_like(qd)
+    c.trace_begin(S * L - 2)                       # capacity smaller than the run: the rest is not recorded
+    for t in range(S):
+        for l in range(L):
+            c.decode_layer_step(t, l, qd[t, l], outs[t, l])
+    tr = c.trace_end()
+    assert tr.shape == (S * L - 2, 6)
+    assert tr[0, 0] >= 0.0
+    assert np.all(np.diff(tr[:, :4], axis=1) >= 0.0)          # points 0..3 are ordered within a call
+    assert np.all(np.diff(tr[:, 0]) >= 0.0)                    # calls are ordered on the compute stream
+    assert np.all(tr[:, 5] > tr[:, 4])                         # a gather takes time
+    for n in range(len(tr) - depth):
+        assert tr[n, 5] <= tr[n + depth, 1] + 1.0              # its slot is attended `depth` calls later
+    assert np.all(tr[:, 4] >= tr[:, 2] - 1.0)                  # and it starts only after this call released the slot
+    c.close()
+
+
 def test_call_order_is_checked(dd):
     w = wl.small(wl.CONFIGS[2], n_layers=2, batch=1, ctx=16 * 40, budget=16 * 4)
     inp = _inputs(w, 1, ragged=False)
