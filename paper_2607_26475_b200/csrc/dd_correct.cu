@@ -115,7 +115,7 @@ int dd_launch_diff(dd_ctx* ctx, const int* pred, const int* truth, int slot, int
 int dd_launch_gather_fix(dd_ctx* ctx, const void* kv_dev, int slot, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
   const size_t per_slot = (size_t)c.batch * c.n_kv_heads * c.k_pages;
-  const int ctas = c.gather_ctas > 0 ? c.gather_ctas : 32;
+  const int ctas = c.gather_ctas > 0 ? c.gather_ctas : 16;
   dd_gather_fix_kernel<<<ctas, 256, 0, st>>>((const char*)kv_dev, ctx->fix_list + slot * per_slot, ctx->fix_count + slot,
                                              ctx->ring + (size_t)slot * ctx->slot_bytes, c.max_pages, c.k_pages,
                                              ctx->err_word);

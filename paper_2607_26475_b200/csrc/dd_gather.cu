@@ -154,7 +154,7 @@ int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int*
                                                                          c.n_kv_heads, c.max_pages, c.k_pages, total,
                                                                          ctx->err_word);
   } else {
-    int ctas = c.gather_ctas > 0 ? c.gather_ctas : 32;
+    int ctas = c.gather_ctas > 0 ? c.gather_ctas : 16;
     const int max_ctas = (total + 7) / 8;
     if (ctas > max_ctas) ctas = max_ctas;
     dd_gather_loads_kernel<<<ctas, 256, 0, st>>>((const char*)kv_dev, idx, n_pages, slot, c.n_kv_heads, c.max_pages,
