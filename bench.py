@@ -401,6 +401,23 @@ def main():
         "pipeline_trace": pipeline_trace,
     }
 
+    if w.structure in ("needle_q", "needle_topic"):
+        # plausibility statistic, not a gate: share of the planted needles' pages inside the set that the
+        # speculated token of (step 0, layer 0) selects
+        ctx.sync()
+        sel = torch.empty((B, w.n_kv_heads, w.k_pages), dtype=torch.int32, device="cuda")
+        ctx.select_topk_chunked(wl.queries(w, 0, 0).cuda(), 1, store.landmarks[0], store.n_pages_dev, store.ctx_len_dev, sel)
+        torch.cuda.synchronize()
+        sel = sel.cpu()
+        hit = tot = 0
+        for b in range(B):
+            pages = wl.needle_positions(w, 0, b) // w.page_tokens
+            for g in range(w.n_kv_heads):
+                chosen = set(sel[b, g].tolist())
+                want = set(pages[g].tolist())
+                hit += len(want & chosen)
+                tot += len(want)
+        line["needle_page_recall"] = hit / max(1, tot)
     if miss is not None:
         line["miss_correction"] = {"missing_pages": miss[0], "selected_pages": miss[1],
                                    "miss_rate": miss[0] / max(1, miss[1]),

@@ -208,6 +208,14 @@ def kv_slab(w: Workload, layer: int, b: int, device="cpu") -> torch.Tensor:
     return slab
 
 
+def needle_positions(w: Workload, layer: int, b: int) -> torch.Tensor:
+    """Token positions [Hkv, n_needles] of the needles `kv_slab` plants in a needle workload (same draws)."""
+    if w.structure not in ("needle_q", "needle_topic"):
+        raise ValueError("not a needle workload")
+    gc = _gen("cpu", w.seed, 23, layer, b)
+    return torch.stack([torch.randperm(w.ctx, generator=gc)[: w.n_needles] for _ in range(w.n_kv_heads)])
+
+
 def ctx_lens(w: Workload, ragged: bool = False) -> torch.Tensor:
     """Context length of every request [B] int32. `ragged` shortens the requests
     unequally (to non-multiples of the page size) for the parity tests."""

@@ -39,8 +39,9 @@ def test_config1_needles_are_four_times_the_normalised_query_direction():
     for g in range(8):
         qm = q[4 * g:4 * g + 4].mean(0)
         needle = (4.0 * qm / qm.norm()).to(torch.bfloat16).float()
-        hits = (keys[g] == needle).all(dim=-1).sum().item()
-        assert hits == 8
+        hits = (keys[g] == needle).all(dim=-1)
+        assert hits.sum().item() == 8
+        assert sorted(hits.nonzero().flatten().tolist()) == sorted(wl.needle_positions(w, 0, 0)[g].tolist())
 
 
 def test_zipf_planted_tokens_crowd_the_recent_end():
