@@ -103,3 +103,27 @@ def test_pipeline_with_two_chunks_per_page(dd):
             want, _ = orc.sparse_decode_attn(f32(q_steps[t, l]), slot, idxs[t][l], ctx_len.numpy(), T)
             check_attention(outs[t, l], want)
     cx.close()
+
+
+def test_chunked_selection_on_long_requests_with_forced_pages(dd):
+    """Config 4's per-request shape (8192 pages, 256 selected, 8 forced) with four landmarks per page and a context
+    that ends inside a page: several blocks per cluster, 64 KiB of logits per block."""
+    B, P, k, forced, c = 1, 8192, 256, 8, 4
+    R = T // c
+    g = torch.Generator().manual_seed(9)
+    lm = torch.randn(B, HKV, P * R, D, generator=g).to(torch.bfloat16)
+    q = torch.randn(B, 2, HQ, D, generator=g).to(torch.bfloat16)
+    ctx_len = torch.tensor([P * T - 9], dtype=torch.int32)        # the last page has two of its four chunks
+    npg = torch.tensor([P], dtype=torch.int32)
+    n_chunks = ((ctx_len + c - 1) // c).numpy()
+    lm[:, :, int(n_chunks[0]):] = 50.0                            # chunks that do not exist must not matter
+    cx = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, forced_recent_pages=forced, landmark_chunk_tokens=c)
+    idx = torch.empty((B, HKV, k), dtype=torch.int32, device="cuda")
+    sc = torch.empty((B, HKV, P), dtype=torch.float32, device="cuda")
+    cx.select_topk_chunked(q.cuda(), 1, lm.cuda(), npg.cuda(), ctx_len.cuda(), idx, sc)
+    assert cx.device_error() == (0, 0)
+    _, want_sc = orc.select_topk(f32(q)[:, 1], f32(lm), npg.numpy(), k, forced, chunks_per_page=R, n_chunks=n_chunks)
+    np.testing.assert_allclose(sc.cpu().numpy()[0], want_sc[0], rtol=2e-4)
+    for h in range(HKV):
+        check_selection(idx.cpu().numpy()[0, h], want_sc[0][h], k, forced)
+    cx.close()
