@@ -201,6 +201,16 @@ int dd_prime(dd_ctx* ctx, const void* q_init);
  *   out  dev bf16 [B][Tq][Hq][d], written */
 int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out);
 
+/* One whole decode step from host buffers: copies the step's queries of all layers from pinned host memory to
+ * the device, runs dd_decode_layer_step for layer 0..L-1, and copies the outputs back, all on the compute stream
+ * (the KV pages come from the bound host store as always). Asynchronous: out_host is complete once the compute
+ * stream has drained (dd_sync, or an event the caller records on that stream after the call).
+ *   q_host    pinned bf16 [L][B][Tq][Hq][d], read when the copy executes
+ *   out_host  pinned bf16 [L][B][Tq][Hq][d], written
+ * The device staging for q and out is part of the context's scratch. Steps follow the same order rule as
+ * dd_decode_layer_step (all layers of `step`, starting at step 0 after dd_prime). */
+int dd_decode_step_host(dd_ctx* ctx, int step, const void* q_host, void* out_host);
+
 /* ---- dual-token causal tail (Sec. 5.2 "Dual-token decoding") ----------------------------------------- */
 
 /* The same attention with the step's own new KV entries appended: the output token and the speculated token

@@ -35,7 +35,7 @@ EXPORTS = [
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
     "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices",
     "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
-    "dd_trace_begin", "dd_trace_end", "dd_trace_read",
+    "dd_trace_begin", "dd_trace_end", "dd_trace_read", "dd_decode_step_host",
 ]
 
 
@@ -96,6 +96,7 @@ def _load() -> C.CDLL:
     lib.dd_fetch_missing_from_host.argtypes = [vp, vp, ip, vp]
     lib.dd_get_merged_indices.argtypes = [vp, ip, C.POINTER(vp)]
     lib.dd_miss_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), C.POINTER(C.c_ulonglong), ip]
+    lib.dd_decode_step_host.argtypes = [vp, ip, vp, vp]
     lib.dd_trace_begin.argtypes = [vp, ip]
     lib.dd_trace_end.argtypes = [vp, C.POINTER(ip)]
     lib.dd_trace_read.argtypes = [vp, ip, ip, vp]
@@ -309,6 +310,10 @@ class Context:
 
     def probe_select_loads(self, landmarks, n_pages, stream=None):
         self._check(lib.dd_probe_select_loads(self._h, _ptr(landmarks), _ptr(n_pages), _stream(stream)))
+
+    def decode_step_host(self, step, q_host, out_host):
+        """One whole step from pinned host tensors [L, B, Tq, Hq, d] (asynchronous on the compute stream)."""
+        self._check(lib.dd_decode_step_host(self._h, step, _ptr(q_host), _ptr(out_host)))
 
     def get_indices(self, step_parity, layer) -> torch.Tensor:
         """A copy of the index set [B, Hkv, k] int32 used at (step parity, layer) (synchronises)."""

@@ -100,10 +100,10 @@ static int dd_resolve_splits(const dd_config* c, int sm_count, int* cluster_out)
 
 struct dd_sizes {
   size_t score_s, score_part, topk_keys, part_o, part_ml, ticket, idx_tab, err, idx_true, idx_merged, fix_stage, fix_list,
-      fix_count, stats;
+      fix_count, stats, stage;
   size_t total() const {
     return score_s + score_part + topk_keys + part_o + part_ml + ticket + idx_tab + err + idx_true + idx_merged +
-           fix_stage + fix_list + fix_count + stats;
+           fix_stage + fix_list + fix_count + stats + 2 * stage;
   }
 };
 
@@ -128,6 +128,7 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
   z.fix_list = up256(D * sel * 16);
   z.fix_count = 256;
   z.stats = 256;
+  z.stage = up256((size_t)c->n_layers * B * c->n_q_tokens * Hq * DD_D * 2);
   return z;
 }
 
@@ -227,7 +228,9 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   ctx->fix_stage = (int2*)base;                      base += z.fix_stage;
   ctx->fix_list = (int4*)base;                       base += z.fix_list;
   ctx->fix_count = (unsigned int*)base;              base += z.fix_count;
-  ctx->miss_stats = (unsigned long long*)base;
+  ctx->miss_stats = (unsigned long long*)base;       base += z.stats;
+  ctx->stage_q = (__nv_bfloat16*)base;               base += z.stage;
+  ctx->stage_out = (__nv_bfloat16*)base;
   DD_CREATE_TRY(cudaMemset(ctx->attn_ticket, 0, z.ticket));
   DD_CREATE_TRY(cudaMemset(ctx->idx_tab, 0, z.idx_tab));
   DD_CREATE_TRY(cudaMemset(ctx->err_word, 0, z.err));
@@ -588,6 +591,29 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
 
 extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out) {
   return dd_layer_step_impl(ctx, step, layer, q, nullptr, nullptr, out);
+}
+
+extern "C" int dd_decode_step_host(dd_ctx* ctx, int step, const void* q_host, void* out_host) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_decode_step_host: ctx is NULL");
+  if (!ctx->primed) return dd_fail(ctx, DD_ERR_STATE, "dd_decode_step_host: call dd_bind and dd_prime first");
+  const dd_config& c = ctx->cfg;
+  for (int i = 0; i < 2; ++i) {                  // both host buffers must be page-locked: the copies are asynchronous
+    const void* p = i == 0 ? q_host : (const void*)out_host;
+    if (!p) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_decode_step_host: host buffer is NULL");
+    cudaPointerAttributes a;
+    cudaError_t e = cudaPointerGetAttributes(&a, p);
+    if (e != cudaSuccess) { cudaGetLastError(); return dd_fail(ctx, DD_ERR_INVALID_ARG, "%s", cudaGetErrorString(e)); }
+    if (a.type != cudaMemoryTypeHost)
+      return dd_fail(ctx, DD_ERR_NOT_PINNED, "dd_decode_step_host: %s must be page-locked host memory", i == 0 ? "q_host" : "out_host");
+  }
+  cudaStream_t cs = (cudaStream_t)c.compute_stream;
+  const size_t per_layer = (size_t)c.batch * c.n_q_tokens * c.n_q_heads * DD_D;
+  const size_t bytes = per_layer * c.n_layers * sizeof(__nv_bfloat16);
+  DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, cs));
+  for (int l = 0; l < c.n_layers; ++l)
+    DD_TRY(dd_layer_step_impl(ctx, step, l, ctx->stage_q + l * per_layer, nullptr, nullptr, ctx->stage_out + l * per_layer));
+  DD_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, ctx->stage_out, bytes, cudaMemcpyDeviceToHost, cs));
+  return DD_OK;
 }
 
 extern "C" int dd_decode_layer_step_causal(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new,

@@ -39,6 +39,8 @@ struct dd_ctx {
   unsigned int* attn_ticket;  // [B*Hkv] arrival counters, zero between launches
   int* idx_tab;          // [2][L][B][Hkv][k]
   int* err_word;         // [2]: code, detail
+  __nv_bfloat16* stage_q;    // [L][B][Tq][Hq][d] device staging of dd_decode_step_host
+  __nv_bfloat16* stage_out;  // [L][B][Tq][Hq][d]
   // miss correction
   int* idx_true;         // [B][Hkv][k] true index of the layer being corrected
   int* idx_merged;       // [D][B][Hkv][k] page held by every position of a slot after the repair

@@ -172,6 +172,29 @@ def test_timeline_of_the_layer_steps(dd):
     c.close()
 
 
+def test_whole_step_from_host_buffers(dd):
+    """dd_decode_step_host gives the same bits as the layer-by-layer calls on device tensors."""
+    S = 2
+    w = wl.small(wl.CONFIGS[2], n_layers=3, batch=2, ctx=16 * 60, budget=16 * 8)
+    inp = _inputs(w, S)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    want, _ = _run(dd, w, S, inp, depth=2, read_idx=False)
+    c = dd.Context(n_layers=w.n_layers, batch=w.batch, max_pages=w.n_pages, k_pages=w.k_pages)
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qh = q_steps.pin_memory()
+    oh = torch.zeros_like(q_steps).pin_memory()
+    for t in range(S):
+        c.decode_step_host(t, qh[t], oh[t])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    assert np.array_equal(raw16(oh), raw16(want))
+    with pytest.raises(dd.DDError) as e:
+        c.decode_step_host(S, q_steps[0].clone(), oh[0])          # pageable queries
+    assert e.value.code == dd.DD_ERR_NOT_PINNED
+    c.close()
+
+
 def test_call_order_is_checked(dd):
     w = wl.small(wl.CONFIGS[2], n_layers=2, batch=1, ctx=16 * 40, budget=16 * 4)
     inp = _inputs(w, 1, ragged=False)
