@@ -17,6 +17,7 @@
  *   - all kernel entry points are asynchronous on the stream they are given (or on the
  *     context's streams for the pipelined calls); dd_create, dd_destroy, dd_sync and
  *     dd_device_error synchronise.
+ *   - timelines, probes, counters and test hooks live in dd_bench.h; they are not part of the method.
  *   - the scratch memory of a context is shared by its calls: calls of the same kind must
  *     be stream-ordered with respect to each other (the pipelined path does this itself).
  *   - tensors are dense, row-major in the index order written; bf16 tensors 16-byte aligned,
@@ -48,6 +49,9 @@ extern "C" {
 
 #define DD_GATHER_LOADS  0          /* zero-copy: warps read the pinned pages with 16-byte loads */
 #define DD_GATHER_BULK   1          /* bulk-copy engine: pinned page -> shared memory -> slot (cp.async.bulk) */
+#define DD_GATHER_STAGED 2          /* the device's copy engine moves runs of adjacent selected pages (or aligned
+                                       blocks) into a staging region, an assembly kernel places them in the slot;
+                                       short runs are read by the zero-copy kernel at the same time */
 
 #define DD_SELECT_AUTO         0    /* fused cluster kernel when the request fits, else the two-kernel path */
 #define DD_SELECT_TWO_KERNELS  1    /* scoring kernel + top-k kernel with logits in global scratch */
@@ -79,6 +83,10 @@ typedef struct dd_config {
   void* urgent_stream;       /* cudaStream_t, ideally of higher priority than copy_stream; used for the missing pages */
   void* select_stream;       /* optional cudaStream_t: the pipelined calls run the next-step selection there, concurrently
                                 with attention (the two are independent); NULL = on the compute stream */
+  int stage_min_run_pages;   /* DD_GATHER_STAGED: runs of at least this many adjacent selected pages go through the
+                                copy engine, shorter ones through the zero-copy kernel; 0 = library default (8) */
+  int stage_block_pages;     /* DD_GATHER_STAGED: 0 = copy exactly the selected runs; 2, 4, 8, 16 or 32 = copy every
+                                aligned block of that many pages that holds a selected page (over-fetch, no stragglers) */
 } dd_config;
 
 /* ---- context ------------------------------------------------------------------------------- */
@@ -93,14 +101,17 @@ int dd_destroy(dd_ctx* ctx);
 size_t dd_slot_bytes(const dd_config* cfg);
 size_t dd_ring_bytes(const dd_config* cfg);
 size_t dd_scratch_bytes(const dd_config* cfg);
-/* Device address of ring slot `slot` (0 <= slot < D). For tests and statistics. */
-int dd_slot_ptr(dd_ctx* ctx, int slot, void** dev_out);
 const char* dd_strerror(int code);
 const char* dd_last_error_message(dd_ctx* ctx);
 /* Synchronises the context's streams (bounded by timeout_s), then reads and clears the device
  * error word. *code is DD_OK, DD_ERR_INDEX_RANGE or DD_ERR_WAIT_EXPIRED; *detail is the
  * offending value (first bad index, or the id of the wait that gave up). */
 int dd_device_error(dd_ctx* ctx, double timeout_s, int* code, int* detail);
+/* The same error word without any synchronisation, enqueue or clearing: a kernel that reports an error also
+ * writes it to a page-locked mirror the host can read at any time, so this call is safe between launches of a
+ * running pipeline. It shows the first error reported since the last dd_device_error (which clears both copies);
+ * an error of a kernel that has not run yet is not visible yet. */
+int dd_last_device_error(dd_ctx* ctx, int* code, int* detail);
 /* Host wait on both context streams with a deadline: DD_ERR_TIMEOUT instead of hanging. */
 int dd_sync(dd_ctx* ctx, double timeout_s);
 
@@ -153,7 +164,12 @@ int dd_select_topk_chunked(dd_ctx* ctx, const void* q, int q_token, const void* 
  *   idx            dev int32 [B][Hkv][k]
  *   n_pages        dev int32 [B] or NULL; when given, idx outside [0, n_pages[b]) is clamped
  *                  and reported (otherwise checked against P)
- *   slot           ring slot number, 0 <= slot < D */
+ *   slot           ring slot number, 0 <= slot < D
+ * With DD_GATHER_STAGED (the copy-engine form of Sec. 5.4: selected KV blocks are moved into a GPU staging
+ * region and a GPU kernel compacts and reorders them into the attention layout) the host needs the index set:
+ * this stand-alone call copies idx to the host and waits for `stream` before it issues the copies; the
+ * pipelined calls copy every selected set to page-locked host memory right after its selection, a whole step
+ * before it is needed. Index checks then happen on the host, with the same clamping and error code. */
 int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, const int* idx, const int* n_pages,
                            int slot, void* stream);
 
@@ -246,37 +262,6 @@ int dd_diff_indices(dd_ctx* ctx, const int* pred_idx, const int* true_idx, int s
 int dd_fetch_missing_from_host(dd_ctx* ctx, const void* host_kv_layer, int slot, void* stream);
 /* Device address of the repaired page list [B][Hkv][k] of ring slot `slot` (valid after a corrected layer step). */
 int dd_get_merged_indices(dd_ctx* ctx, int slot, const int** dev_idx);
-/* Synchronises, then reports how many pages were missing and how many were selected since the last reset. */
-int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset);
-
-/* ---- timeline of the pipelined calls ------------------------------------------------------------------ */
-
-/* dd_trace_begin arms a timeline of up to max_layer_steps calls of dd_decode_layer_step (it creates timing
- * events; no device memory). Every traced call records six points, in microseconds since the first traced call:
- *   [0] the compute stream reaches the layer step (all earlier compute work done)
- *   [1] every transfer the layer needs is complete: attention starts ([1] - [0] = time the compute stream
- *       was stalled on the host link, plus the true-index selection and diff under miss correction)
- *   [2] attention done (buffer released)
- *   [3] end of the layer step on the compute stream (selection done or rejoined)
- *   [4] the gather this call enqueued (layer + ring depth) starts on the copy stream, its waits satisfied
- *   [5] that gather is complete
- * dd_trace_end stops recording, synchronises and returns the number of traced calls; dd_trace_read copies
- * `count` rows of 6 floats starting at row `first` into host memory `out`. DD_ERR_STATE when no trace exists. */
-#define DD_TRACE_FIELDS 6
-int dd_trace_begin(dd_ctx* ctx, int max_layer_steps);
-int dd_trace_end(dd_ctx* ctx, int* n_recorded);
-int dd_trace_read(dd_ctx* ctx, int first, int count, float* out);
-
-/* ---- measurement aids ------------------------------------------------------------------------------- */
-
-/* Load-only twins of the two HBM-bound kernels: the same grid, the same walk over pages / landmark rows and the
- * same 16-byte fragment loads as dd_sparse_decode_attn (over ring slot `slot`) and as the fused selection
- * (over `landmarks`, dev bf16 [B][Hkv][P*R][d], with n_pages dev int32 [B]), but no arithmetic, no exchange and
- * no output. Their duration is what the memory system delivers for that launch shape and size; the benchmark
- * reports it next to the kernels' own times. dd_probe_select_loads needs the fused selection path
- * (DD_ERR_STATE otherwise). Asynchronous on `stream`. */
-int dd_probe_attn_loads(dd_ctx* ctx, int slot, void* stream);
-int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const int* n_pages, void* stream);
 
 /* ---- attention without any allocation ----------------------------------------------------------- */
 
@@ -299,6 +284,8 @@ int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const int* n_pages
  *     clears the arrival counters it needs on `stream` before the kernel. Two calls that overlap on the
  *     GPU (different streams, no ordering between them) race on the array and give wrong results:
  *     order them.
+ *   - Every tensor pointer is checked on the host before anything is enqueued (cudaPointerGetAttributes,
+ *     which allocates nothing): host memory or another device's memory gives DD_ERR_INVALID_ARG.
  * Asynchronous on `stream`. Returns DD_OK or DD_ERR_INVALID_ARG / DD_ERR_CUDA; the message is
  * available from dd_last_error_message(NULL) on the calling thread. */
 size_t dd_static_scratch_capacity(void);

@@ -1,0 +1,86 @@
+/* dd_bench.h — instrumentation of the sparse decode library: timelines, load-only probes, counters and test
+ * hooks used by the benchmark and the tests. None of these calls is a step of the method and none has a
+ * counterpart in the paper; the method's boundary is dd.h. Same conventions as dd.h.
+ */
+#ifndef DD_BENCH_H_
+#define DD_BENCH_H_
+
+#include "dd.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Device address of ring slot `slot` (0 <= slot < D): lets a test read back what a gather wrote. */
+int dd_slot_ptr(dd_ctx* ctx, int slot, void** dev_out);
+
+/* ---- miss statistics --------------------------------------------------------------------------------- */
+
+/* Synchronises, then reports how many pages were missing and how many were selected since the last reset. */
+int dd_miss_stats(dd_ctx* ctx, unsigned long long* missing, unsigned long long* selected, int reset);
+
+/* ---- timeline of the pipelined calls ------------------------------------------------------------------ */
+
+/* dd_trace_begin arms a timeline of up to max_layer_steps calls of dd_decode_layer_step (it creates timing
+ * events; no device memory). Every traced call records eight points, in microseconds since the first traced call:
+ *   [0] the compute stream reaches the layer step (all earlier compute work done)
+ *   [1] every transfer the layer needs is complete: attention starts ([1] - [0] = time the compute stream
+ *       was stalled on the host link, plus the true-index selection and diff under miss correction)
+ *   [2] attention done (buffer released)
+ *   [3] end of the layer step on the compute stream (selection done or rejoined)
+ *   [4] the gather this call enqueued (layer + ring depth) starts on the copy stream, its waits satisfied
+ *   [5] that gather is complete
+ *   [6] under miss correction: the fetch of this layer's missing pages starts on the urgent stream (the
+ *       prefetch of the slot and the repair list are complete); -1 without miss correction
+ *   [7] under miss correction: that fetch is complete; -1 without miss correction
+ * dd_trace_end stops recording, synchronises and returns the number of traced calls; dd_trace_read copies
+ * `count` rows of DD_TRACE_FIELDS floats starting at row `first` into host memory `out`. DD_ERR_STATE when no trace exists. */
+#define DD_TRACE_FIELDS 8
+int dd_trace_begin(dd_ctx* ctx, int max_layer_steps);
+int dd_trace_end(dd_ctx* ctx, int* n_recorded);
+int dd_trace_read(dd_ctx* ctx, int first, int count, float* out);
+
+/* ---- measurement aids ------------------------------------------------------------------------------- */
+
+/* Load-only twins of the two HBM-bound kernels: the same grid, the same walk over pages / landmark rows and the
+ * same 16-byte fragment loads as dd_sparse_decode_attn (over ring slot `slot`) and as the fused selection
+ * (over `landmarks`, dev bf16 [B][Hkv][P*R][d], with n_pages dev int32 [B]), but no arithmetic, no exchange and
+ * no output. Their duration is what the memory system delivers for that launch shape and size; the benchmark
+ * reports it next to the kernels' own times. dd_probe_select_loads needs the fused selection path
+ * (DD_ERR_STATE otherwise). Asynchronous on `stream`. */
+int dd_probe_attn_loads(dd_ctx* ctx, int slot, void* stream);
+int dd_probe_select_loads(dd_ctx* ctx, const void* landmarks, const int* n_pages, void* stream);
+
+/* ---- counters of the staged gather ---------------------------------------------------------------- */
+
+/* Totals since the context was created (or since the last call with reset != 0) over all gathers issued in
+ * DD_GATHER_STAGED mode; host-side counters, no synchronisation:
+ *   out[0] gathers, out[1] copy-engine copies issued, out[2] bytes those copies moved over the host link,
+ *   out[3] selected pages that went through the staging region, out[4] selected pages read by the zero-copy
+ *   kernel, out[5] microseconds the host spent waiting for index sets, out[6] microseconds the host spent
+ *   forming runs and issuing copies. */
+#define DD_GATHER_STATS_FIELDS 7
+int dd_gather_stats(dd_ctx* ctx, unsigned long long* out, int reset);
+
+/* ---- test hooks ------------------------------------------------------------------------------------- */
+
+/* Limit of the bounded device-side waits of the bulk gather engine (default 2 s), and a way to make one run
+ * out without faulting anything: with inflate_first_stage != 0 the first stage of block 0 expects 16 bytes
+ * more than its copy delivers, so its wait can never complete; the copy itself lands normally, the wait gives
+ * up after wait_seconds, the block waits (bounded) for its other copies in flight and returns, and the device
+ * error word reports DD_ERR_WAIT_EXPIRED. For tests of that error path only. */
+int dd_set_bulk_wait(dd_ctx* ctx, double wait_seconds, int inflate_first_stage);
+
+/* The cluster-size search of the fused selection kernel with the device queries replaced by a callback, so that
+ * it can be tested without a GPU: returns the chosen blocks per (request, KV head), or 0 when no cluster size
+ * fits (the two-kernel path is then used). fits(blocks, shared_bytes, user) says whether clusters of that many
+ * blocks with that much dynamic shared memory per block can be resident; allow16 says whether 16-block
+ * (non-portable) clusters may be tried. rows_per_page = landmarks per page, group = query heads per KV head. */
+int dd_test_pick_cluster(int max_pages, int problems, int sm_count, int rows_per_page, int group, int allow16,
+                         int (*fits)(int blocks, size_t shared_bytes, void* user), void* user, int* pages_per_block,
+                         size_t* shared_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* DD_BENCH_H_ */

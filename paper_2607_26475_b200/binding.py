@@ -1,4 +1,5 @@
-"""Thin ctypes binding of the C-ABI library (`include/dd.h`): argument marshalling only.
+"""Thin ctypes binding of the C-ABI library (`include/dd.h`, instrumentation in `include/dd_bench.h`):
+argument marshalling only.
 
 Every step of the path runs in the library's CUDA kernels. torch is used for device and
 pinned memory and for streams; tensors are passed as raw pointers. There is no CPU
@@ -25,6 +26,9 @@ DD_ERR_STATE = -6
 DD_ERR_WAIT_EXPIRED = -7
 DD_GATHER_LOADS = 0
 DD_GATHER_BULK = 1
+DD_GATHER_STAGED = 2
+DD_GATHER_STATS_FIELDS = 7
+DD_TRACE_FIELDS = 8
 DD_SELECT_AUTO = 0
 DD_SELECT_TWO_KERNELS = 1
 
@@ -35,7 +39,8 @@ EXPORTS = [
     "dd_decode_layer_step", "dd_get_indices", "dd_static_scratch_capacity", "dd_sparse_decode_attn_static",
     "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices",
     "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
-    "dd_trace_begin", "dd_trace_end", "dd_trace_read", "dd_decode_step_host",
+    "dd_trace_begin", "dd_trace_end", "dd_trace_read", "dd_decode_step_host", "dd_last_device_error",
+    "dd_gather_stats", "dd_set_bulk_wait", "dd_test_pick_cluster",
 ]
 
 
@@ -49,7 +54,7 @@ class DDConfig(C.Structure):
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
         ("landmark_chunk_tokens", C.c_int), ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
-        ("select_stream", C.c_void_p),
+        ("select_stream", C.c_void_p), ("stage_min_run_pages", C.c_int), ("stage_block_pages", C.c_int),
     ]
 
 
@@ -57,6 +62,9 @@ class DDError(RuntimeError):
     def __init__(self, code: int, message: str):
         super().__init__(f"dd error {code}: {message}")
         self.code = code
+
+
+PICK_FITS = C.CFUNCTYPE(C.c_int, C.c_int, C.c_size_t, C.c_void_p)
 
 
 def _load() -> C.CDLL:
@@ -102,6 +110,10 @@ def _load() -> C.CDLL:
     lib.dd_trace_read.argtypes = [vp, ip, ip, vp]
     lib.dd_probe_attn_loads.argtypes = [vp, ip, vp]
     lib.dd_probe_select_loads.argtypes = [vp, vp, vp, vp]
+    lib.dd_last_device_error.argtypes = [vp, C.POINTER(ip), C.POINTER(ip)]
+    lib.dd_gather_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), ip]
+    lib.dd_set_bulk_wait.argtypes = [vp, C.c_double, ip]
+    lib.dd_test_pick_cluster.argtypes = [ip, ip, ip, ip, ip, ip, PICK_FITS, vp, C.POINTER(ip), C.POINTER(C.c_size_t)]
     lib.dd_static_scratch_capacity.argtypes = []
     lib.dd_static_scratch_capacity.restype = C.c_size_t
     lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7
@@ -161,7 +173,8 @@ class Context:
     def __init__(self, *, n_layers, batch, max_pages, k_pages, n_q_heads=32, n_kv_heads=8, head_dim=128,
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
                  gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None,
-                 miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0, select_stream=None):
+                 miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0, select_stream=None,
+                 stage_min_run_pages=0, stage_block_pages=0):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
@@ -176,7 +189,8 @@ class Context:
                             _ptr(ring), ring.numel() * ring.element_size() if ring is not None else 0,
                             landmark_chunk_tokens, 1 if miss_correction else 0,
                             self.urgent_stream.cuda_stream if self.urgent_stream is not None else None,
-                            select_stream.cuda_stream if select_stream is not None else None)
+                            select_stream.cuda_stream if select_stream is not None else None,
+                            stage_min_run_pages, stage_block_pages)
         self.select_stream = select_stream
         self._h = C.c_void_p()
         self._keep = []
@@ -230,6 +244,22 @@ class Context:
         code, detail = C.c_int(), C.c_int()
         self._check(lib.dd_device_error(self._h, timeout_s, C.byref(code), C.byref(detail)))
         return code.value, detail.value
+
+    def last_device_error(self):
+        """(code, detail) of the first device-side error since the last device_error(), without synchronising."""
+        code, detail = C.c_int(), C.c_int()
+        self._check(lib.dd_last_device_error(self._h, C.byref(code), C.byref(detail)))
+        return code.value, detail.value
+
+    def gather_stats(self, reset=False) -> dict:
+        """Host-side counters of the staged gather (see dd_gather_stats)."""
+        a = (C.c_ulonglong * DD_GATHER_STATS_FIELDS)()
+        self._check(lib.dd_gather_stats(self._h, a, 1 if reset else 0))
+        names = ("gathers", "copies", "copied_bytes", "pages_staged", "pages_zero_copy", "host_wait_us", "host_issue_us")
+        return dict(zip(names, [int(x) for x in a]))
+
+    def set_bulk_wait(self, wait_seconds: float, inflate_first_stage: bool = False):
+        self._check(lib.dd_set_bulk_wait(self._h, wait_seconds, 1 if inflate_first_stage else 0))
 
     # -- entry points
     def build_landmarks(self, kv_layer, ctx_len, landmarks, stream=None):
@@ -296,11 +326,12 @@ class Context:
         self._check(lib.dd_trace_begin(self._h, max_layer_steps))
 
     def trace_end(self):
-        """Stops the trace and returns it as a [n, 6] float32 numpy array of microseconds (see dd_trace_begin)."""
+        """Stops the trace and returns it as a [n, DD_TRACE_FIELDS] float32 numpy array of microseconds (see
+        dd_trace_begin in dd_bench.h)."""
         import numpy as np
         n = C.c_int()
         self._check(lib.dd_trace_end(self._h, C.byref(n)))
-        out = np.zeros((n.value, 6), dtype=np.float32)
+        out = np.zeros((n.value, DD_TRACE_FIELDS), dtype=np.float32)
         if n.value:
             self._check(lib.dd_trace_read(self._h, 0, n.value, out.ctypes.data_as(C.c_void_p)))
         return out

@@ -6,6 +6,7 @@
 #include <chrono>
 #include <new>
 #include <thread>
+#include <vector>
 
 #include "dd_common.cuh"
 
@@ -55,7 +56,13 @@ static const char* dd_check_config(const dd_config* c) {
   if (c->k_pages < 1 || c->k_pages > c->max_pages) return "need 1 <= k_pages <= max_pages";
   if (c->forced_recent_pages < 0 || c->forced_recent_pages > c->k_pages) return "need 0 <= forced_recent_pages <= k_pages";
   if (c->ring_depth < 2 || c->ring_depth > DD_MAX_RING) return "ring_depth must be in [2, 8]";
-  if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK) return "unknown gather_mode";
+  if (c->gather_mode != DD_GATHER_LOADS && c->gather_mode != DD_GATHER_BULK && c->gather_mode != DD_GATHER_STAGED)
+    return "unknown gather_mode";
+  if (c->stage_min_run_pages < 0) return "stage_min_run_pages must be >= 0";
+  {
+    const int bp = c->stage_block_pages;
+    if (bp != 0 && bp != 2 && bp != 4 && bp != 8 && bp != 16 && bp != 32) return "stage_block_pages must be 0, 2, 4, 8, 16 or 32";
+  }
   if (c->select_mode != DD_SELECT_AUTO && c->select_mode != DD_SELECT_TWO_KERNELS) return "unknown select_mode";
   if (c->gather_ctas < 0 || c->attn_splits < 0) return "gather_ctas and attn_splits must be >= 0";
   if (c->miss_correction != 0 && c->miss_correction != 1) return "miss_correction must be 0 or 1";
@@ -162,6 +169,23 @@ static void dd_free_all(dd_ctx* ctx) {
     if (ctx->urgent_done[i]) cudaEventDestroy(ctx->urgent_done[i]);
   }
   if (ctx->q_ready) cudaEventDestroy(ctx->q_ready);
+  if (ctx->err_host) cudaFreeHost(ctx->err_host);
+  if (ctx->idx_host) cudaFreeHost(ctx->idx_host);
+  if (ctx->staging) cudaFree(ctx->staging);
+  for (int i = 0; i < DD_STAGE_LISTS; ++i) {
+    if (ctx->list_host[i]) cudaFreeHost(ctx->list_host[i]);
+    if (ctx->list_free[i]) cudaEventDestroy(ctx->list_free[i]);
+  }
+  if (ctx->aux_fork) cudaEventDestroy(ctx->aux_fork);
+  if (ctx->aux_join) cudaEventDestroy(ctx->aux_join);
+  if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
+  if (ctx->idx_copied) {
+    for (int l = 0; l < ctx->cfg.n_layers; ++l)
+      if (ctx->idx_copied[l]) cudaEventDestroy(ctx->idx_copied[l]);
+    delete[] ctx->idx_copied;
+  }
+  delete[] ctx->n_pages_host;
+  delete[] ctx->host_kv_orig;
   if (ctx->sel_done) {
     for (int l = 0; l < ctx->cfg.n_layers; ++l)
       if (ctx->sel_done[l]) cudaEventDestroy(ctx->sel_done[l]);
@@ -234,6 +258,15 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   DD_CREATE_TRY(cudaMemset(ctx->attn_ticket, 0, z.ticket));
   DD_CREATE_TRY(cudaMemset(ctx->idx_tab, 0, z.idx_tab));
   DD_CREATE_TRY(cudaMemset(ctx->err_word, 0, z.err));
+  {
+    // page-locked mirror of the error word; its device-visible address sits behind the two words
+    DD_CREATE_TRY(cudaHostAlloc((void**)&ctx->err_host, 2 * sizeof(int), cudaHostAllocMapped));
+    ctx->err_host[0] = ctx->err_host[1] = 0;
+    void* mirror_dev = nullptr;
+    DD_CREATE_TRY(cudaHostGetDevicePointer(&mirror_dev, ctx->err_host, 0));
+    DD_CREATE_TRY(cudaMemcpy(ctx->err_word + 2, &mirror_dev, sizeof(void*), cudaMemcpyHostToDevice));
+  }
+  ctx->bulk_wait_ns = 2000000000ull;
   DD_CREATE_TRY(cudaMemset(ctx->fix_count, 0, z.fix_count));
   DD_CREATE_TRY(cudaMemset(ctx->miss_stats, 0, z.stats));
   if (cfg->ring_mem) {
@@ -265,6 +298,29 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
     DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->sel_done[l], cudaEventDisableTiming));
   ctx->landmarks = new const void*[cfg->n_layers]();
   ctx->host_kv = new const void*[cfg->n_layers]();
+  ctx->host_kv_orig = new const void*[cfg->n_layers]();
+  if (cfg->gather_mode == DD_GATHER_STAGED) {
+    const size_t total = (size_t)cfg->batch * cfg->n_kv_heads * cfg->k_pages;
+    ctx->stage_min_run = cfg->stage_min_run_pages > 0 ? cfg->stage_min_run_pages : 8;
+    ctx->stage_block = cfg->stage_block_pages;
+    ctx->staging_pages = total * (size_t)(ctx->stage_block > 0 ? ctx->stage_block : 1);
+    DD_CREATE_TRY(cudaMalloc(&ctx->staging, ctx->staging_pages * DD_PAGE_BYTES));
+    DD_CREATE_TRY(cudaHostAlloc((void**)&ctx->idx_host, (size_t)2 * cfg->n_layers * total * sizeof(int), cudaHostAllocDefault));
+    ctx->n_pages_host = new int[cfg->batch]();
+    ctx->idx_copied = new cudaEvent_t[cfg->n_layers]();
+    for (int l = 0; l < cfg->n_layers; ++l)
+      DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->idx_copied[l], cudaEventDisableTiming));
+    for (int i = 0; i < DD_STAGE_LISTS; ++i) {
+      DD_CREATE_TRY(cudaHostAlloc((void**)&ctx->list_host[i], (ctx->staging_pages + total) * sizeof(int), cudaHostAllocMapped));
+      void* dv = nullptr;
+      DD_CREATE_TRY(cudaHostGetDevicePointer(&dv, ctx->list_host[i], 0));
+      ctx->list_dev[i] = (const int*)dv;
+      DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->list_free[i], cudaEventDisableTiming));
+    }
+    DD_CREATE_TRY(cudaStreamCreateWithFlags(&ctx->aux_stream, cudaStreamNonBlocking));
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->aux_fork, cudaEventDisableTiming));
+    DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->aux_join, cudaEventDisableTiming));
+  }
   int rc = dd_select_setup(ctx);
   if (rc == DD_OK) rc = dd_gather_setup(ctx);
   if (rc != DD_OK) {
@@ -281,8 +337,10 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
 extern "C" int dd_sync(dd_ctx* ctx, double timeout_s) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sync: ctx is NULL");
   const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(timeout_s);
-  cudaStream_t streams[4] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream, nullptr, nullptr};
+  cudaStream_t streams[5] = {(cudaStream_t)ctx->cfg.compute_stream, (cudaStream_t)ctx->cfg.copy_stream, nullptr, nullptr,
+                             nullptr};
   int n_streams = 2;
+  if (ctx->aux_stream) streams[n_streams++] = ctx->aux_stream;
   if (ctx->cfg.miss_correction) streams[n_streams++] = (cudaStream_t)ctx->cfg.urgent_stream;
   if (ctx->cfg.select_stream) streams[n_streams++] = (cudaStream_t)ctx->cfg.select_stream;
   for (int i = 0; i < n_streams; ++i) {
@@ -314,8 +372,21 @@ extern "C" int dd_device_error(dd_ctx* ctx, double timeout_s, int* code, int* de
   DD_CUDA_TRY(ctx, cudaDeviceSynchronize());       // standalone calls may have used other streams
   DD_CUDA_TRY(ctx, cudaMemcpy(w, ctx->err_word, sizeof(w), cudaMemcpyDeviceToHost));
   DD_CUDA_TRY(ctx, cudaMemset(ctx->err_word, 0, sizeof(w)));
+  if (w[0] == 0 && ctx->host_err[0] != 0) { w[0] = ctx->host_err[0]; w[1] = ctx->host_err[1]; }   // host-side index checks
+  ctx->host_err[0] = ctx->host_err[1] = 0;
+  ctx->err_host[0] = ctx->err_host[1] = 0;
   if (code) *code = w[0];
   if (detail) *detail = w[1];
+  return DD_OK;
+}
+
+extern "C" int dd_last_device_error(dd_ctx* ctx, int* code, int* detail) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_last_device_error: ctx is NULL");
+  const volatile int* m = ctx->err_host;
+  int c = m[0], d = m[1];
+  if (c == 0 && ctx->host_err[0] != 0) { c = ctx->host_err[0]; d = ctx->host_err[1]; }
+  if (code) *code = c;
+  if (detail) *detail = d;
   return DD_OK;
 }
 
@@ -420,6 +491,17 @@ extern "C" int dd_gather_kv_from_host(dd_ctx* ctx, const void* host_kv_layer, co
   DD_TRY(dd_check_store(ctx, host_kv_layer, "host_kv_layer", &kv_dev));
   DD_TRY(dd_check_dev(ctx, idx, "idx", 4));
   if (n_pages) DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
+  if (ctx->cfg.gather_mode == DD_GATHER_STAGED) {
+    // the host forms the runs: bring the index set over and wait for it
+    const size_t total = (size_t)ctx->cfg.batch * ctx->cfg.n_kv_heads * ctx->cfg.k_pages;
+    std::vector<int> idx_h(total), np_h(n_pages ? ctx->cfg.batch : 0);
+    DD_CUDA_TRY(ctx, cudaMemcpyAsync(idx_h.data(), idx, total * sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    if (n_pages)
+      DD_CUDA_TRY(ctx, cudaMemcpyAsync(np_h.data(), n_pages, np_h.size() * sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    DD_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+    return dd_launch_gather_staged(ctx, host_kv_layer, kv_dev, idx_h.data(), idx, n_pages ? np_h.data() : nullptr, n_pages,
+                                   ctx->ring + (size_t)slot * ctx->slot_bytes, (cudaStream_t)stream);
+  }
   return dd_launch_gather(ctx, kv_dev, idx, n_pages, ctx->ring + (size_t)slot * ctx->slot_bytes, (cudaStream_t)stream);
 }
 
@@ -452,11 +534,14 @@ extern "C" int dd_bind(dd_ctx* ctx, const void* const* landmarks_per_layer, cons
     DD_TRY(dd_check_store(ctx, host_kv_per_layer[l], "host_kv_per_layer[l]", &dv));
     ctx->landmarks[l] = landmarks_per_layer[l];
     ctx->host_kv[l] = dv;
+    ctx->host_kv_orig[l] = host_kv_per_layer[l];
   }
   DD_TRY(dd_check_dev(ctx, n_pages, "n_pages", 4));
   DD_TRY(dd_check_dev(ctx, ctx_len, "ctx_len", 4));
   ctx->n_pages = n_pages;
   ctx->ctx_len = ctx_len;
+  if (ctx->n_pages_host)       // the staged gather checks indices on the host
+    DD_CUDA_TRY(ctx, cudaMemcpy(ctx->n_pages_host, n_pages, ctx->cfg.batch * sizeof(int), cudaMemcpyDeviceToHost));
   ctx->bound = true;
   return DD_OK;
 }
@@ -464,6 +549,20 @@ extern "C" int dd_bind(dd_ctx* ctx, const void* const* landmarks_per_layer, cons
 static int* dd_idx_of(dd_ctx* ctx, int parity, int layer) {
   const dd_config& c = ctx->cfg;
   return ctx->idx_tab + ((size_t)(parity & 1) * c.n_layers + layer) * c.batch * c.n_kv_heads * c.k_pages;
+}
+
+// What follows every selection of a set the pipeline will gather: in staged mode the set is copied to page-locked
+// host memory on the stream that selected it; then the "selection done" event of the layer is recorded.
+static int dd_after_select(dd_ctx* ctx, int parity, int layer, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  if (c.gather_mode == DD_GATHER_STAGED) {
+    const size_t per_set = (size_t)c.batch * c.n_kv_heads * c.k_pages;
+    DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->idx_host + ((size_t)(parity & 1) * c.n_layers + layer) * per_set,
+                                     dd_idx_of(ctx, parity, layer), per_set * sizeof(int), cudaMemcpyDeviceToHost, st));
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->idx_copied[layer], st));
+  }
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], st));
+  return DD_OK;
 }
 
 // Gather number n = step * L + layer goes to slot n % D. It may start once the attention that last
@@ -476,8 +575,18 @@ static int dd_enqueue_gather(dd_ctx* ctx, long long n, cudaEvent_t ev_start = nu
   if (ctx->released_recorded[slot]) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->released[slot], 0));
   DD_CUDA_TRY(ctx, cudaStreamWaitEvent(xs, ctx->sel_done[layer], 0));
   if (ev_start) DD_CUDA_TRY(ctx, cudaEventRecord(ev_start, xs));
-  DD_TRY(dd_launch_gather(ctx, ctx->host_kv[layer], dd_idx_of(ctx, step, layer), ctx->n_pages,
-                          ctx->ring + (size_t)slot * ctx->slot_bytes, xs));
+  if (c.gather_mode == DD_GATHER_STAGED) {
+    // the set was copied to the host right after its selection (normally a whole step ago)
+    DD_TRY(dd_wait_index_copy(ctx, layer));
+    const size_t per_set = (size_t)c.batch * c.n_kv_heads * c.k_pages;
+    DD_TRY(dd_launch_gather_staged(ctx, ctx->host_kv_orig[layer], ctx->host_kv[layer],
+                                   ctx->idx_host + ((size_t)(step & 1) * c.n_layers + layer) * per_set,
+                                   dd_idx_of(ctx, step, layer), ctx->n_pages_host, ctx->n_pages,
+                                   ctx->ring + (size_t)slot * ctx->slot_bytes, xs));
+  } else {
+    DD_TRY(dd_launch_gather(ctx, ctx->host_kv[layer], dd_idx_of(ctx, step, layer), ctx->n_pages,
+                            ctx->ring + (size_t)slot * ctx->slot_bytes, xs));
+  }
   if (ev_end) DD_CUDA_TRY(ctx, cudaEventRecord(ev_end, xs));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->ready[slot], xs));
   return DD_OK;
@@ -495,17 +604,19 @@ extern "C" int dd_prime(dd_ctx* ctx, const void* q_init) {
   for (int l = 0; l < c.n_layers; ++l) {
     DD_TRY(dd_launch_select(ctx, (const __nv_bfloat16*)q_init + l * q_layer, 0, 1, ctx->landmarks[l], ctx->n_pages,
                             dd_idx_of(ctx, 0, l), nullptr, cs, ctx->ctx_len));
-    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[l], cs));
+    DD_TRY(dd_after_select(ctx, 0, l, cs));
   }
   for (int i = 0; i < DD_MAX_RING; ++i) ctx->released_recorded[i] = false;
   const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
+  ctx->primed = false;
   for (long long n = 0; n < ahead; ++n) DD_TRY(dd_enqueue_gather(ctx, n));
   ctx->next_call = 0;
+  ctx->in_flight = false;
   ctx->primed = true;
   return DD_OK;
 }
 
-static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new, const void* v_new,
+static int dd_layer_step_body(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new, const void* v_new,
                               void* out) {
   if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_decode_layer_step: ctx is NULL");
   if (!ctx->primed) return dd_fail(ctx, DD_ERR_STATE, "dd_decode_layer_step: call dd_bind and dd_prime first");
@@ -521,7 +632,8 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   if (k_new) DD_TRY(dd_check_dev(ctx, v_new, "v_new"));
   cudaStream_t cs = (cudaStream_t)c.compute_stream;
   const int slot = (int)(n % c.ring_depth);
-  cudaEvent_t* tr = nullptr;                     // this call's six timeline events, when a trace is armed
+  ctx->in_flight = true;                         // from here on a failure leaves the ring protocol out of step
+  cudaEvent_t* tr = nullptr;                     // this call's timeline events, when a trace is armed
   if (ctx->trace_on && ctx->trace_n < ctx->trace_cap) {
     tr = ctx->trace_ev + (size_t)ctx->trace_n * DD_TRACE_FIELDS;
     if (ctx->trace_n == 0) DD_CUDA_TRY(ctx, cudaEventRecord(ctx->trace_origin, cs));
@@ -542,7 +654,7 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(ss, ctx->q_ready, 0));
     DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
                             dd_idx_of(ctx, step + 1, layer), nullptr, sel_st, ctx->ctx_len));
-    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], sel_st));
+    DD_TRY(dd_after_select(ctx, step + 1, layer, sel_st));
   }
   if (c.miss_correction) {
     // true index from the current token, repair list, missing pages on the urgent stream; the selection for
@@ -555,12 +667,14 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->fix_ready[slot], cs));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->fix_ready[slot], 0));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(us, ctx->ready[slot], 0));                  // the prefetch wrote the slot first
+    if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[6], us));
     DD_TRY(dd_launch_gather_fix(ctx, ctx->host_kv[layer], slot, us));
+    if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[7], us));
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->urgent_done[slot], us));
     if (!side_select) {
       DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
                               dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
-      DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+      DD_TRY(dd_after_select(ctx, step + 1, layer, cs));
     }
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->ready[slot], 0));
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->urgent_done[slot], 0));            // all transfers of the layer complete
@@ -577,7 +691,7 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   if (!c.miss_correction && !side_select) {
     DD_TRY(dd_launch_select(ctx, q, spec_token, c.n_q_tokens, ctx->landmarks[layer], ctx->n_pages,
                             dd_idx_of(ctx, step + 1, layer), nullptr, cs, ctx->ctx_len));
-    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->sel_done[layer], cs));
+    DD_TRY(dd_after_select(ctx, step + 1, layer, cs));
   }
   if (side_select) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(cs, ctx->sel_done[layer], 0));   // q may be reused after this call
   // the slot just released takes the gather `ahead` layers further on (index set known: it was
@@ -586,7 +700,20 @@ static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, c
   const int ahead = c.ring_depth < c.n_layers ? c.ring_depth : c.n_layers;
   DD_TRY(dd_enqueue_gather(ctx, n + ahead, tr ? tr[4] : nullptr, tr ? tr[5] : nullptr));
   ctx->next_call = n + 1;
+  ctx->in_flight = false;
   return DD_OK;
+}
+
+// A failure after the call began to enqueue work cannot be undone (events are recorded, index tables may be
+// overwritten): the context then needs dd_prime again.
+static int dd_layer_step_impl(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new, const void* v_new,
+                              void* out) {
+  const int rc = dd_layer_step_body(ctx, step, layer, q, k_new, v_new, out);
+  if (rc != DD_OK && ctx && ctx->in_flight) {
+    ctx->primed = false;
+    ctx->in_flight = false;
+  }
+  return rc;
 }
 
 extern "C" int dd_decode_layer_step(dd_ctx* ctx, int step, int layer, const void* q, void* out) {
@@ -609,11 +736,20 @@ extern "C" int dd_decode_step_host(dd_ctx* ctx, int step, const void* q_host, vo
   cudaStream_t cs = (cudaStream_t)c.compute_stream;
   const size_t per_layer = (size_t)c.batch * c.n_q_tokens * c.n_q_heads * DD_D;
   const size_t bytes = per_layer * c.n_layers * sizeof(__nv_bfloat16);
-  DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, cs));
-  for (int l = 0; l < c.n_layers; ++l)
-    DD_TRY(dd_layer_step_impl(ctx, step, l, ctx->stage_q + l * per_layer, nullptr, nullptr, ctx->stage_out + l * per_layer));
-  DD_CUDA_TRY(ctx, cudaMemcpyAsync(out_host, ctx->stage_out, bytes, cudaMemcpyDeviceToHost, cs));
-  return DD_OK;
+  if ((long long)step * c.n_layers != ctx->next_call)
+    return dd_fail(ctx, DD_ERR_STATE, "expected step %lld, layer %lld next, got step %d", ctx->next_call / c.n_layers,
+                   ctx->next_call % c.n_layers, step);
+  // once the first copy is queued the step cannot be taken back: any later failure needs dd_prime again
+  cudaError_t e = cudaMemcpyAsync(ctx->stage_q, q_host, bytes, cudaMemcpyHostToDevice, cs);
+  int rc = e == cudaSuccess ? DD_OK : dd_fail(ctx, DD_ERR_CUDA, "cudaMemcpyAsync(q_host): %s", cudaGetErrorString(e));
+  for (int l = 0; l < c.n_layers && rc == DD_OK; ++l)
+    rc = dd_layer_step_impl(ctx, step, l, ctx->stage_q + l * per_layer, nullptr, nullptr, ctx->stage_out + l * per_layer);
+  if (rc == DD_OK) {
+    e = cudaMemcpyAsync(out_host, ctx->stage_out, bytes, cudaMemcpyDeviceToHost, cs);
+    if (e != cudaSuccess) rc = dd_fail(ctx, DD_ERR_CUDA, "cudaMemcpyAsync(out_host): %s", cudaGetErrorString(e));
+  }
+  if (rc != DD_OK) ctx->primed = false;
+  return rc;
 }
 
 extern "C" int dd_decode_layer_step_causal(dd_ctx* ctx, int step, int layer, const void* q, const void* k_new,
@@ -736,9 +872,28 @@ extern "C" int dd_trace_read(dd_ctx* ctx, int first, int count, float* out) {
   for (int i = 0; i < count; ++i) {
     for (int f = 0; f < DD_TRACE_FIELDS; ++f) {
       float ms = 0.f;
+      if (f >= 6 && !ctx->cfg.miss_correction) {   // urgent-stream points exist under miss correction only
+        out[(size_t)i * DD_TRACE_FIELDS + f] = -1.f;
+        continue;
+      }
       DD_CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->trace_origin, ctx->trace_ev[(size_t)(first + i) * DD_TRACE_FIELDS + f]));
       out[(size_t)i * DD_TRACE_FIELDS + f] = ms * 1e3f;
     }
   }
+  return DD_OK;
+}
+
+extern "C" int dd_gather_stats(dd_ctx* ctx, unsigned long long* out, int reset) {
+  if (!ctx || !out) return dd_fail(ctx, DD_ERR_INVALID_ARG, "dd_gather_stats: NULL argument");
+  for (int i = 0; i < DD_GATHER_STATS_FIELDS; ++i) out[i] = ctx->gstats[i];
+  if (reset) memset(ctx->gstats, 0, sizeof(ctx->gstats));
+  return DD_OK;
+}
+
+extern "C" int dd_set_bulk_wait(dd_ctx* ctx, double wait_seconds, int inflate_first_stage) {
+  if (!ctx) return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_set_bulk_wait: ctx is NULL");
+  if (!(wait_seconds > 0.0) || wait_seconds > 60.0) return dd_fail(ctx, DD_ERR_INVALID_ARG, "wait_seconds must be in (0, 60]");
+  ctx->bulk_wait_ns = (unsigned long long)(wait_seconds * 1e9);
+  ctx->bulk_inflate = inflate_first_stage ? 1 : 0;
   return DD_OK;
 }

@@ -18,8 +18,6 @@
 
 #include "dd_common.cuh"
 
-DD_TRACE_DECLARE(dd_trace_attn)
-#define DD_TRACE_MARK(i) DD_TRACE_MARK_IN(dd_trace_attn, i)
 
 constexpr int ATTN_WARPS = 4;
 constexpr int ATTN_THREADS = ATTN_WARPS * 32;
@@ -86,7 +84,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
   __shared__ float2 blk_ml[ATTN_ROWS];
   __shared__ int sm_last;
 
-  DD_TRACE_MARK(0);
   // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G)
   uint4 qf[4];
   if (gl < n_rows) {
@@ -220,11 +217,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     }
     softmax_pv(acc);
     if (has_next) dd_load_v(vbase + (size_t)jn * DD_HALF_PAGE_BYTES, gl, t, v);
-    if (j == p_begin + warp) DD_TRACE_MARK(1);
     page = page_next;
     j = jn;
   }
-  DD_TRACE_MARK(2);
   // l over the 8 row groups of the warp
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -260,7 +255,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     blk_ml[n] = make_float2(M, L);
   }
   __syncthreads();
-  DD_TRACE_MARK(3);
   const int d = threadIdx.x;                     // one channel per thread, all rows
   float ob[ATTN_ROWS];
 #pragma unroll
@@ -333,7 +327,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
     }
     if (n_groups > 1) __threadfence();
     cl.sync();                                   // nobody leaves while its shared memory may still be read
-    DD_TRACE_MARK(4);
     if (n_groups == 1 || rank != 0) return;
   } else {
     // ---- one block per cluster: publish the block's partial directly
@@ -509,6 +502,25 @@ static size_t dd_static_need(int batch, int n_kv_heads, int n_splits, size_t* of
 
 extern "C" size_t dd_static_scratch_capacity(void) { return DD_STATIC_SCRATCH_BYTES; }
 
+// Host-side pointer check of the context-free entry point: device (or managed) memory of the current device,
+// aligned for its element type. cudaPointerGetAttributes allocates nothing.
+static int dd_static_check_dev(const void* p, const char* what, int align, int dev) {
+  if (((uintptr_t)p) & (uintptr_t)(align - 1))
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: %s is not %d-byte aligned", what, align);
+  cudaPointerAttributes a;
+  const cudaError_t e = cudaPointerGetAttributes(&a, p);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: %s: %s", what, cudaGetErrorString(e));
+  }
+  if (a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: %s is not device memory", what);
+  if (a.type == cudaMemoryTypeDevice && a.device != dev)
+    return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: %s lives on device %d, the current device is %d",
+                   what, a.device, dev);
+  return DD_OK;
+}
+
 extern "C" int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_heads, int head_dim, int page_tokens,
                                             int k_pages, int n_q_tokens, int n_splits, const void* q,
                                             const void* slot, const int* idx, const int* ctx_len, void* out,
@@ -536,6 +548,15 @@ extern "C" int dd_sparse_decode_attn_static(int batch, int n_q_heads, int n_kv_h
   if (e != cudaSuccess) return dd_fail(nullptr, DD_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
   if (dev < 0 || dev >= DD_STATIC_MAX_DEVICES)
     return dd_fail(nullptr, DD_ERR_INVALID_ARG, "dd_sparse_decode_attn_static: device ordinal %d not supported", dev);
+  {
+    int rc;
+    if ((rc = dd_static_check_dev(q, "q", 16, dev)) != DD_OK) return rc;
+    if ((rc = dd_static_check_dev(slot, "slot", 16, dev)) != DD_OK) return rc;
+    if ((rc = dd_static_check_dev(idx, "idx", 4, dev)) != DD_OK) return rc;
+    if ((rc = dd_static_check_dev(ctx_len, "ctx_len", 4, dev)) != DD_OK) return rc;
+    if ((rc = dd_static_check_dev(out, "out", 16, dev)) != DD_OK) return rc;
+    if (out_lse && (rc = dd_static_check_dev(out_lse, "out_lse", 4, dev)) != DD_OK) return rc;
+  }
   unsigned char* base = nullptr;
   {
     std::lock_guard<std::mutex> lock(g_static_scratch_mutex);

@@ -7,6 +7,7 @@
 #include <stdio.h>
 
 #include "../../include/dd.h"
+#include "../../include/dd_bench.h"
 
 constexpr int DD_D = 128;          // head_dim the kernels are written for
 constexpr int DD_T = 16;           // tokens per page
@@ -15,6 +16,7 @@ constexpr int DD_HALF_PAGE_BYTES = DD_T * DD_ROW_BYTES;   // K (or V) part of a 
 constexpr int DD_PAGE_BYTES = 2 * DD_HALF_PAGE_BYTES;     // 8 KiB
 constexpr int DD_MAX_RING = 8;
 constexpr int DD_SCORE_TILE = 128; // pages scored by one thread block
+constexpr int DD_STAGE_LISTS = 8;  // page-locked descriptor buffers of the staged gather (host may run this far ahead)
 
 struct dd_ctx {
   dd_config cfg;
@@ -38,7 +40,9 @@ struct dd_ctx {
   float2* attn_part_ml;  // [B][Hkv][S][8] (max, sum) in the log2 domain
   unsigned int* attn_ticket;  // [B*Hkv] arrival counters, zero between launches
   int* idx_tab;          // [2][L][B][Hkv][k]
-  int* err_word;         // [2]: code, detail
+  int* err_word;         // [0] code, [1] detail, [2..3] device-visible address of err_host
+  int* err_host;         // page-locked mirror [2] that reporting kernels also write (read without synchronising)
+  int host_err[2];       // errors found by host-side index checks (staged gather)
   __nv_bfloat16* stage_q;    // [L][B][Tq][Hq][d] device staging of dd_decode_step_host
   __nv_bfloat16* stage_out;  // [L][B][Tq][Hq][d]
   // miss correction
@@ -61,10 +65,30 @@ struct dd_ctx {
   // bound tables
   const void** landmarks;  // [L]
   const void** host_kv;    // [L] device-visible addresses
+  const void** host_kv_orig;  // [L] the pointers as given to dd_bind (sources of copy-engine copies)
   const int* n_pages;
   const int* ctx_len;
   bool bound, primed;
   long long next_call;     // step * L + layer expected by dd_decode_layer_step
+  bool in_flight;          // a pipelined call has begun to enqueue work (a failure now needs dd_prime again)
+  // bulk gather engine: limit of its bounded waits, and the test hook that makes one run out
+  unsigned long long bulk_wait_ns;
+  int bulk_inflate;
+  // staged gather (DD_GATHER_STAGED)
+  int stage_min_run, stage_block;
+  int* idx_host;           // page-locked [2][L][B*Hkv*k]: every selected set, copied right after its selection
+  cudaEvent_t* idx_copied; // [L] that copy is complete
+  int* n_pages_host;       // [B]
+  char* staging;           // device landing zone of the copy engine, staging_pages pages of 8 KiB
+  size_t staging_pages;
+  int* list_host[DD_STAGE_LISTS];   // page-locked: [staging_pages] staged page -> slot item (or -1), then [B*Hkv*k] straggler items
+  const int* list_dev[DD_STAGE_LISTS];
+  cudaEvent_t list_free[DD_STAGE_LISTS];
+  bool list_used[DD_STAGE_LISTS];
+  long long list_next;
+  cudaStream_t aux_stream; // library-owned: the zero-copy kernel of the short runs, next to the copy engine
+  cudaEvent_t aux_fork, aux_join;
+  unsigned long long gstats[DD_GATHER_STATS_FIELDS];
   // optional timeline of the pipelined calls: DD_TRACE_FIELDS timing events per layer step
   cudaEvent_t* trace_ev;
   cudaEvent_t trace_origin;
@@ -85,6 +109,11 @@ int dd_launch_build_landmarks(dd_ctx* ctx, const void* kv_dev, const int* ctx_le
 int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_tensor, const void* landmarks,
                      const int* n_pages, int* out_idx, float* out_scores, cudaStream_t st, const int* ctx_len = nullptr);
 int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int* n_pages, char* slot, cudaStream_t st);
+// Staged gather of one layer: idx_h is the index set on the host (already complete), kv_src the store as given by
+// the caller; copies run on `st`, the short runs on the context's auxiliary stream (joined into `st` before return).
+int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev, const int* idx_h, const int* idx_dev,
+                            const int* n_pages_h, const int* n_pages_dev, char* slot, cudaStream_t st);
+int dd_wait_index_copy(dd_ctx* ctx, int layer);   // host wait (bounded) until layer's newest index set is on the host
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
                    float* out_lse, cudaStream_t st, const void* k_new = nullptr, const void* v_new = nullptr);
 int dd_launch_attn_loads_only(dd_ctx* ctx, const char* slot, cudaStream_t st);
@@ -97,9 +126,18 @@ int dd_launch_gather_fix(dd_ctx* ctx, const void* kv_dev, int slot, cudaStream_t
 // ---------------------------------------------------------------------------------------------
 #ifdef __CUDACC__
 
-// First error wins; later ones are dropped. Never traps.
+// First error wins; later ones are dropped. Never traps. The winner also writes the page-locked mirror whose
+// address the host stored behind the two words.
 __device__ __forceinline__ void dd_report(int* err_word, int code, int detail) {
-  if (atomicCAS(err_word, 0, code) == 0) err_word[1] = detail;
+  if (atomicCAS(err_word, 0, code) == 0) {
+    err_word[1] = detail;
+    volatile int* mirror = *reinterpret_cast<int* volatile*>(err_word + 2);
+    if (mirror) {
+      mirror[1] = detail;
+      __threadfence_system();
+      mirror[0] = code;
+    }
+  }
 }
 
 // 16-byte read-only load that does not allocate in L1 (every byte on this path is used once per block).
@@ -135,26 +173,5 @@ __device__ __forceinline__ void dd_ml_merge(float& m, float& l, float m2, float 
   l = l * a + l2 * b;
   m = mn;
 }
-
-// Optional per-block timeline for tuning (compile with -DDD_TRACE; never in the shipped library): mark i of
-// block (x, y, z) is the global nanosecond timer when thread 0 passed it; <name>_read copies the table out.
-#ifdef DD_TRACE
-#define DD_TRACE_DECLARE(name)                                                                       \
-  __device__ unsigned long long name[1 << 16][8];                                                    \
-  extern "C" int name##_read(unsigned long long* host, size_t bytes) {                               \
-    return (int)cudaMemcpyFromSymbol(host, name, bytes);                                             \
-  }
-#define DD_TRACE_MARK_IN(name, i)                                                                    \
-  do {                                                                                               \
-    if (threadIdx.x == 0) {                                                                          \
-      unsigned long long t__;                                                                        \
-      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t__));                                        \
-      name[(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x][i] = t__;                 \
-    }                                                                                                \
-  } while (0)
-#else
-#define DD_TRACE_DECLARE(name)
-#define DD_TRACE_MARK_IN(name, i)
-#endif
 
 #endif  // __CUDACC__

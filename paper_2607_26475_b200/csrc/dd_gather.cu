@@ -7,6 +7,13 @@
 // reads in flight per warp across the host link), then sixteen stores.
 // DD_GATHER_BULK: one thread per block drives the bulk-copy engine: page -> shared memory ring
 // (cp.async.bulk with mbarrier completion) -> two bulk stores into the slot. Every wait is bounded.
+// DD_GATHER_STAGED: the host, which holds a copy of the index set, forms runs of adjacent selected pages and
+// lets the device's copy engine move each long run with one asynchronous copy into a staging region; an
+// assembly kernel places the staged pages in the slot, and the short runs are read by the zero-copy kernel on
+// a second stream at the same time.
+#include <chrono>
+#include <vector>
+
 #include "dd_common.cuh"
 
 __device__ __forceinline__ int dd_checked_page(const int* idx, const int* n_pages, int item, int b, int P,
@@ -54,7 +61,6 @@ __global__ void __launch_bounds__(256) dd_gather_loads_kernel(const char* __rest
 // Bulk-copy engine variant
 // ------------------------------------------------------------------------------------------------
 constexpr int BULK_STAGES = 16;                       // 16 x 8 KiB = 128 KiB of shared memory per block
-constexpr unsigned long long BULK_WAIT_NS = 2000000000ull;   // a wait gives up after two seconds
 
 __device__ __forceinline__ uint32_t dd_smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -64,10 +70,10 @@ __device__ __forceinline__ unsigned long long dd_globaltimer() {
   return t;
 }
 
-__device__ __forceinline__ bool dd_mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool dd_mbar_wait_bounded(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
   const unsigned long long t0 = dd_globaltimer();
   for (unsigned it = 0;; ++it) {
-    if ((it & 63u) == 63u && dd_globaltimer() - t0 > BULK_WAIT_NS) return false;
+    if ((it & 63u) == 63u && dd_globaltimer() - t0 > limit_ns) return false;
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -82,7 +88,8 @@ __device__ __forceinline__ bool dd_mbar_wait_bounded(uint32_t bar, uint32_t pari
 
 __global__ void __launch_bounds__(32) dd_gather_bulk_kernel(const char* __restrict__ kv, const int* __restrict__ idx,
                                                             const int* __restrict__ n_pages, char* __restrict__ slot,
-                                                            int Hkv, int P, int k, int total, int* err_word) {
+                                                            int Hkv, int P, int k, int total, int* err_word,
+                                                            unsigned long long wait_ns, int inflate) {
   extern __shared__ __align__(128) unsigned char stage_mem[];     // BULK_STAGES pages
   __shared__ __align__(8) unsigned long long full_bar[BULK_STAGES];
   if (threadIdx.x != 0) return;                       // one thread drives the engine; no block-wide barrier is used
@@ -100,8 +107,9 @@ __global__ void __launch_bounds__(32) dd_gather_bulk_kernel(const char* __restri
     const int s = n % BULK_STAGES;
     const uint32_t bar = dd_smem_addr(&full_bar[s]);
     const uint32_t dst = dd_smem_addr(stage_mem + (size_t)s * DD_PAGE_BYTES);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)DD_PAGE_BYTES)
-                 : "memory");
+    // test hook: the first stage of block 0 may be told to expect more bytes than its copy delivers
+    const uint32_t expect = (uint32_t)DD_PAGE_BYTES + ((inflate && n == 0 && blockIdx.x == 0) ? 16u : 0u);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(expect) : "memory");
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"((uint32_t)DD_PAGE_BYTES), "r"(bar)
                  : "memory");
@@ -114,7 +122,7 @@ __global__ void __launch_bounds__(32) dd_gather_bulk_kernel(const char* __restri
   int n = 0;
   for (; n < n_mine; ++n) {
     const int s = n % BULK_STAGES;
-    if (!dd_mbar_wait_bounded(dd_smem_addr(&full_bar[s]), (uint32_t)((n / BULK_STAGES) & 1))) { ok = false; break; }
+    if (!dd_mbar_wait_bounded(dd_smem_addr(&full_bar[s]), (uint32_t)((n / BULK_STAGES) & 1), wait_ns)) { ok = false; break; }
     const int item = blockIdx.x + n * gridDim.x;
     const int j = item % k, bg = item / k;
     char* dst_k = slot + ((size_t)bg * 2 * k + j) * DD_HALF_PAGE_BYTES;
@@ -139,7 +147,7 @@ __global__ void __launch_bounds__(32) dd_gather_bulk_kernel(const char* __restri
     dd_report(err_word, DD_ERR_WAIT_EXPIRED, 1);
     // loads already issued may still land in shared memory: give each one more bounded wait before leaving
     for (int m = n + 1; m < issued; ++m)
-      dd_mbar_wait_bounded(dd_smem_addr(&full_bar[m % BULK_STAGES]), (uint32_t)((m / BULK_STAGES) & 1));
+      dd_mbar_wait_bounded(dd_smem_addr(&full_bar[m % BULK_STAGES]), (uint32_t)((m / BULK_STAGES) & 1), wait_ns);
   }
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");       // stores complete before the block retires
 }
@@ -152,7 +160,8 @@ int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int*
     if (ctas > total) ctas = total;
     dd_gather_bulk_kernel<<<ctas, 32, BULK_STAGES * DD_PAGE_BYTES, st>>>((const char*)kv_dev, idx, n_pages, slot,
                                                                          c.n_kv_heads, c.max_pages, c.k_pages, total,
-                                                                         ctx->err_word);
+                                                                         ctx->err_word, ctx->bulk_wait_ns,
+                                                                         ctx->bulk_inflate);
   } else {
     int ctas = c.gather_ctas > 0 ? c.gather_ctas : 16;
     const int max_ctas = (total + 7) / 8;
@@ -161,6 +170,180 @@ int dd_launch_gather(dd_ctx* ctx, const void* kv_dev, const int* idx, const int*
                                                  c.k_pages, total, ctx->err_word);
   }
   DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Staged variant: copy engine -> staging region -> assembly kernel; short runs by zero-copy loads
+// ------------------------------------------------------------------------------------------------
+// The zero-copy kernel over a list of slot items (item = unit * k + position) instead of all of them.
+__global__ void __launch_bounds__(256) dd_gather_list_kernel(const char* __restrict__ kv, const int* __restrict__ idx,
+                                                             const int* __restrict__ n_pages,
+                                                             const int* __restrict__ items, int n_items,
+                                                             char* __restrict__ slot, int Hkv, int P, int k,
+                                                             int* err_word) {
+  const int lane = threadIdx.x & 31;
+  const int n_warps = gridDim.x * (blockDim.x >> 5);
+  for (int i = (threadIdx.x >> 5) * gridDim.x + blockIdx.x; i < n_items; i += n_warps) {
+    const int item = items[i];
+    const int j = item % k;
+    const int bg = item / k;
+    const int p = dd_checked_page(idx, n_pages, item, bg / Hkv, P, err_word);
+    const char* src = kv + ((size_t)bg * P + p) * DD_PAGE_BYTES + lane * 16;
+    char* dst_k = slot + ((size_t)bg * 2 * k + j) * DD_HALF_PAGE_BYTES + lane * 16;
+    char* dst_v = dst_k + (size_t)k * DD_HALF_PAGE_BYTES;
+    uint4 r[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) r[q] = dd_ld_stream(src + q * 512);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) dd_st_v4(dst_k + q * 512, r[q]);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) dd_st_v4(dst_v + q * 512, r[8 + q]);
+  }
+}
+
+// Assembly: staged page s (8 KiB: K half, V half) goes to slot item map[s]; map[s] < 0 marks a page that was
+// only fetched because it shares an aligned block with a selected one.
+__global__ void __launch_bounds__(256) dd_assemble_kernel(const char* __restrict__ staging, const int* __restrict__ map,
+                                                          int n_staged, char* __restrict__ slot, int k) {
+  const int lane = threadIdx.x & 31;
+  const int n_warps = gridDim.x * (blockDim.x >> 5);
+  for (int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); s < n_staged; s += n_warps) {
+    const int item = map[s];
+    if (item < 0) continue;
+    const int j = item % k;
+    const int bg = item / k;
+    const char* src = staging + (size_t)s * DD_PAGE_BYTES + lane * 16;
+    char* dst_k = slot + ((size_t)bg * 2 * k + j) * DD_HALF_PAGE_BYTES + lane * 16;
+    char* dst_v = dst_k + (size_t)k * DD_HALF_PAGE_BYTES;
+    uint4 r[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) r[q] = dd_ld_stream(src + q * 512);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) dd_st_v4(dst_k + q * 512, r[q]);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) dd_st_v4(dst_v + q * 512, r[8 + q]);
+  }
+}
+
+// Host wait on an event with a deadline (the staged gather's only blocking points).
+static int dd_wait_event(dd_ctx* ctx, cudaEvent_t ev, double seconds, const char* what) {
+  const auto deadline = std::chrono::steady_clock::now() + std::chrono::duration<double>(seconds);
+  for (;;) {
+    const cudaError_t e = cudaEventQuery(ev);
+    if (e == cudaSuccess) return DD_OK;
+    if (e != cudaErrorNotReady) return dd_fail(ctx, DD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    if (std::chrono::steady_clock::now() > deadline)
+      return dd_fail(ctx, DD_ERR_TIMEOUT, "%s: not complete after %.1f s", what, seconds);
+  }
+}
+
+int dd_wait_index_copy(dd_ctx* ctx, int layer) {
+  const auto t0 = std::chrono::steady_clock::now();
+  const int rc = dd_wait_event(ctx, ctx->idx_copied[layer], 30.0, "staged gather: copy of the index set to the host");
+  ctx->gstats[5] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t0).count();
+  return rc;
+}
+
+int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev, const int* idx_h, const int* idx_dev,
+                            const int* n_pages_h, const int* n_pages_dev, char* slot, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const int Hkv = c.n_kv_heads, P = c.max_pages, k = c.k_pages;
+  const int units = c.batch * Hkv, total = units * k;
+  const int Bp = ctx->stage_block, min_run = ctx->stage_min_run;
+  const int li = (int)(ctx->list_next % DD_STAGE_LISTS);
+  if (ctx->list_used[li]) {
+    const auto tw = std::chrono::steady_clock::now();
+    const int rc = dd_wait_event(ctx, ctx->list_free[li], 30.0, "staged gather: descriptor buffer still in use");
+    ctx->gstats[5] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - tw).count();
+    if (rc != DD_OK) return rc;
+  }
+  const auto t0 = std::chrono::steady_clock::now();
+  int* map = ctx->list_host[li];
+  int* strag = map + ctx->staging_pages;
+  int n_staged = 0, n_strag = 0;
+  unsigned long long n_copies = 0, sel_staged = 0;
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->aux_fork, st));          // the short runs may start when the copies may
+  const char* src_base = (const char*)kv_src;
+  for (int bg = 0; bg < units; ++bg) {
+    int limit = P;
+    if (n_pages_h) limit = n_pages_h[bg / Hkv] < P ? n_pages_h[bg / Hkv] : P;
+    const int* row = idx_h + (size_t)bg * k;
+    auto page_of = [&](int j) {
+      int p = row[j];
+      if (p < 0 || p >= limit) {
+        if (ctx->host_err[0] == 0) { ctx->host_err[0] = DD_ERR_INDEX_RANGE; ctx->host_err[1] = p; }
+        p = p < 0 ? 0 : (limit > 0 ? limit - 1 : 0);
+      }
+      return p;
+    };
+    int j = 0;
+    while (j < k) {
+      const int p = page_of(j);
+      int jj = j + 1, page0, n_pages_copy;
+      if (Bp > 0) {
+        // aligned blocks: extend over the selected pages that fall into this block or the one right after the last
+        int blk_end = p / Bp;
+        while (jj < k) {
+          const int bj = page_of(jj) / Bp;
+          if (bj < blk_end || bj > blk_end + 1 || page_of(jj) <= page_of(jj - 1)) break;
+          blk_end = bj;
+          ++jj;
+        }
+        page0 = (p / Bp) * Bp;
+        const int page1 = (blk_end + 1) * Bp < P ? (blk_end + 1) * Bp : P;
+        n_pages_copy = page1 - page0;
+      } else {
+        while (jj < k && page_of(jj) == p + (jj - j)) ++jj;
+        page0 = p;
+        n_pages_copy = jj - j;
+        if (n_pages_copy < min_run) {
+          for (int x = j; x < jj; ++x) strag[n_strag++] = bg * k + x;
+          j = jj;
+          continue;
+        }
+      }
+      if ((size_t)n_staged + n_pages_copy > ctx->staging_pages)
+        return dd_fail(ctx, DD_ERR_INVALID_ARG, "staged gather: staging region too small (index set not ascending?)");
+      for (int x = 0; x < n_pages_copy; ++x) map[n_staged + x] = -1;
+      for (int x = j; x < jj; ++x) map[n_staged + page_of(x) - page0] = bg * k + x;
+      DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->staging + (size_t)n_staged * DD_PAGE_BYTES,
+                                       src_base + ((size_t)bg * P + page0) * DD_PAGE_BYTES,
+                                       (size_t)n_pages_copy * DD_PAGE_BYTES, cudaMemcpyDefault, st));
+      ++n_copies;
+      sel_staged += (unsigned long long)(jj - j);
+      n_staged += n_pages_copy;
+      j = jj;
+    }
+  }
+  if (n_strag > 0) {
+    int ctas = c.gather_ctas > 0 ? c.gather_ctas : 16;
+    const int max_ctas = (n_strag + 7) / 8;
+    if (ctas > max_ctas) ctas = max_ctas;
+    DD_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->aux_stream, ctx->aux_fork, 0));
+    dd_gather_list_kernel<<<ctas, 256, 0, ctx->aux_stream>>>((const char*)kv_dev, idx_dev, n_pages_dev,
+                                                             ctx->list_dev[li] + ctx->staging_pages, n_strag, slot, Hkv, P,
+                                                             k, ctx->err_word);
+    DD_CUDA_TRY(ctx, cudaGetLastError());
+    DD_CUDA_TRY(ctx, cudaEventRecord(ctx->aux_join, ctx->aux_stream));
+  }
+  if (n_staged > 0) {
+    int blocks = (n_staged + 7) / 8;
+    if (blocks > 4 * ctx->sm_count) blocks = 4 * ctx->sm_count;
+    dd_assemble_kernel<<<blocks, 256, 0, st>>>(ctx->staging, ctx->list_dev[li], n_staged, slot, k);
+    DD_CUDA_TRY(ctx, cudaGetLastError());
+  }
+  if (n_strag > 0) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->aux_join, 0));
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->list_free[li], st));
+  ctx->list_used[li] = true;
+  ++ctx->list_next;
+  ctx->gstats[0] += 1;
+  ctx->gstats[1] += n_copies;
+  ctx->gstats[2] += (unsigned long long)n_staged * DD_PAGE_BYTES;
+  ctx->gstats[3] += sel_staged;
+  ctx->gstats[4] += (unsigned long long)n_strag;
+  ctx->gstats[6] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t0).count();
+  (void)total;
   return DD_OK;
 }
 

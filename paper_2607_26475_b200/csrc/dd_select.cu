@@ -355,8 +355,6 @@ __global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
 // ------------------------------------------------------------------------------------------------
 namespace cg = cooperative_groups;
 
-DD_TRACE_DECLARE(dd_trace_select)
-#define DD_SEL_MARK(i) DD_TRACE_MARK_IN(dd_trace_select, i)
 
 constexpr int SEL_THREADS = 256;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
@@ -431,7 +429,6 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   const int n_local_rows = max(0, min(n_rows_req, (p_lo + ppc) * R) - p_lo * R);
   if (tid == 0) { cta_minmax[0] = 0xFFFFFFFFu; cta_minmax[1] = 0u; cta_cnt[0] = 0u; cta_cnt[1] = 0u; cand_n = 0u; }
 
-  DD_SEL_MARK(0);
   // ---- A. logits of this block's pages (same MMA formulation as dd_score_kernel), kept in shared memory
   float m_run[2] = {-INFINITY, -INFINITY};
   float l_run[2] = {0.f, 0.f};
@@ -511,10 +508,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     for (int w = 1; w < SEL_WARPS; ++w) dd_ml_merge(m, l, red[w][tid].x, red[w][tid].y, false);
     cta_ml[tid] = make_float2(m, l);
   }
-  DD_SEL_MARK(1);
   // ---- B. log-sum-exp of the whole request: every block merges the partials of all blocks
   cl.sync();
-  DD_SEL_MARK(2);
   if (tid < G) {
     float m = -INFINITY, l = 0.f;
     for (int r = 0; r < C; ++r) {
@@ -552,9 +547,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     if (lane == 0) { atomicMin(&cta_minmax[0], kmin); atomicMax(&cta_minmax[1], kmax); }
   }
   const uint32_t* keys = reinterpret_cast<const uint32_t*>(s_sm);      // key of local page pl at keys[pl * KS]
-  DD_SEL_MARK(3);
   cl.sync();
-  DD_SEL_MARK(4);
   uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
   for (int r = 0; r < C; ++r) {
     kmin = min(kmin, *cl.map_shared_rank(&cta_minmax[0], r));
@@ -654,7 +647,6 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       }
     }
   }
-  DD_SEL_MARK(5);
 
   // ---- E. how many pages each block contributes, then ordered compaction of this block's pages
   {
@@ -669,7 +661,6 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     if (lane == 0) { atomicAdd(&cta_cnt[0], gt); atomicAdd(&cta_cnt[1], eq); }
   }
   cl.sync();
-  DD_SEL_MARK(6);
   unsigned base_gt = 0, base_eq = 0;
   for (int r = 0; r < rank; ++r) {
     base_gt += *cl.map_shared_rank(&cta_cnt[0], r);
@@ -697,7 +688,6 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   if (rank == 0)                                 // precondition k <= n_pages violated: pad with the last valid page
     for (int j = k_eff + tid; j < k; j += SEL_THREADS) out[j] = np > 0 ? np - 1 : 0;
   cl.sync();                                     // nobody leaves while its shared memory may still be read
-  DD_SEL_MARK(7);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -791,46 +781,66 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
 // Picks the cluster size of the fused selection: a power of two such that all clusters are resident at once
 // (two blocks per SM), every block has at least 32 pages, and a block's share of the logits fits in shared
 // memory. Up to 8 blocks, 16 for very long requests. 0 = not possible, use the two-kernel path.
+// The search walks a fixed candidate list exactly once, so it always terminates; `fits` answers whether clusters of that shape can be resident on the device.
+extern "C" int dd_test_pick_cluster(int max_pages, int problems, int sm_count, int rows_per_page, int group, int allow16,
+                                    int (*fits)(int blocks, size_t shared_bytes, void* user), void* user,
+                                    int* pages_per_block, size_t* shared_bytes) {
+  if (max_pages < 1 || problems < 1 || sm_count < 1 || rows_per_page < 1 || group < 1 || !fits) return 0;
+  const int c_max = (max_pages >= 32768 && allow16) ? 16 : 8;
+  int start = 1;
+  while (start * 2 <= c_max && (long long)start * 2 * problems <= 2LL * sm_count && max_pages / (start * 2) >= 32) start *= 2;
+  // candidates: the preferred size, every larger one, then the smaller ones (fewer, larger blocks)
+  int cand[16], n_cand = 0;
+  for (int C = start; C <= c_max; C *= 2) cand[n_cand++] = C;
+  for (int C = start / 2; C >= 1; C /= 2) cand[n_cand++] = C;
+  for (int i = 0; i < n_cand; ++i) {
+    const int C = cand[i];
+    int ppc = (max_pages + C - 1) / C;
+    ppc = (ppc + 31) & ~31;                                // whole pairs of MMA tiles
+    const size_t smem = (size_t)ppc * rows_per_page * group * 4 + 2 * RADIX_BINS * 4;
+    if (smem > (size_t)SEL_MAX_SMEM) continue;             // too long for this cluster size
+    if (!fits(C, smem, user)) continue;
+    if (pages_per_block) *pages_per_block = ppc;
+    if (shared_bytes) *shared_bytes = smem;
+    return C;
+  }
+  return 0;
+}
+
+static int dd_select_cluster_fits(int C, size_t smem, void* user) {
+  const dd_ctx* ctx = (const dd_ctx*)user;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(C, ctx->cfg.n_kv_heads, ctx->cfg.batch);
+  cfg.blockDim = dim3(SEL_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n_clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&n_clusters, dd_select_fused_kernel, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return n_clusters >= 1;
+}
+
 static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
   const dd_config& c = ctx->cfg;
-  const int G = ctx->G;
-  const int problems = c.batch * c.n_kv_heads;
   // function attributes are per process, not per context: always ask for the largest the kernel may use
   if (cudaFuncSetAttribute(dd_select_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SEL_MAX_SMEM) !=
       cudaSuccess) { cudaGetLastError(); return 0; }
   const bool big_ok = cudaFuncSetAttribute(dd_select_fused_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed,
                                            1) == cudaSuccess;
   if (!big_ok) cudaGetLastError();
-  const int c_max = (c.max_pages >= 32768 && big_ok) ? 16 : 8;
-  int C = 1;
-  while (C * 2 <= c_max && C * 2 * problems <= 2 * ctx->sm_count && c.max_pages / (C * 2) >= 32) C *= 2;
-  for (; C <= c_max; C *= 2) {
-    int ppc = (c.max_pages + C - 1) / C;
-    ppc = (ppc + 31) & ~31;                                // whole pairs of MMA tiles
-    const size_t smem = (size_t)ppc * ctx->R * G * 4 + 2 * RADIX_BINS * 4;
-    if (smem > (size_t)SEL_MAX_SMEM) continue;             // too long for this cluster size: try a larger one
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(C, c.n_kv_heads, c.batch);
-    cfg.blockDim = dim3(SEL_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = C;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&n_clusters, dd_select_fused_kernel, &cfg) != cudaSuccess || n_clusters < 1) {
-      cudaGetLastError();
-      if (C == 16) { C = 4; continue; }                    // 16-block clusters unavailable: fall back to 8
-      continue;
-    }
-    *ppc_out = ppc;
-    *smem_out = (int)smem;
-    return C;
-  }
-  return 0;
+  size_t smem = 0;
+  const int C = dd_test_pick_cluster(c.max_pages, c.batch * c.n_kv_heads, ctx->sm_count, ctx->R, ctx->G, big_ok ? 1 : 0,
+                                     dd_select_cluster_fits, ctx, ppc_out, &smem);
+  *smem_out = (int)smem;
+  return C;
 }
 
 int dd_select_setup(dd_ctx* ctx) {

@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include "dd.h"
+#include "dd_bench.h"   /* dd_slot_ptr: reads back what the gather wrote */
 
 #define CHECK_DD(expr)                                                                          \
   do {                                                                                          \

@@ -7,7 +7,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared():
-    text = open(os.path.join(ROOT, "include", "dd.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", h)).read() for h in ("dd.h", "dd_bench.h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(dd_[a-z_0-9]+)\s*\(", text)))
 
@@ -20,7 +20,7 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert "dd_select_topk" in names and "dd_gather_kv_from_host" in names
     assert "dd_sparse_decode_attn" in names and "dd_decode_layer_step" in names
     for n in names:
-        assert hasattr(lib, n), f"{n} is declared in include/dd.h but not exported"
+        assert hasattr(lib, n), f"{n} is declared in include/*.h but not exported"
 
 
 def test_binding_lists_the_same_entry_points_and_error_strings():
@@ -31,11 +31,53 @@ def test_binding_lists_the_same_entry_points_and_error_strings():
     assert binding.lib.dd_strerror(0) == b"ok"
     assert binding.lib.dd_strerror(binding.DD_ERR_NOT_PINNED) == b"host memory is not page-locked"
     # size queries and configuration checks run on the host
-    cfg = binding.DDConfig(32, 8, 32, 8, 128, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None)
+    cfg = binding.DDConfig(32, 8, 32, 8, 128, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0)
     assert binding.lib.dd_slot_bytes(ctypes.byref(cfg)) == 64 << 20
     assert binding.lib.dd_ring_bytes(ctypes.byref(cfg)) == 128 << 20
-    bad = binding.DDConfig(32, 8, 32, 8, 64, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None)
+    bad = binding.DDConfig(32, 8, 32, 8, 64, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0)
     assert binding.lib.dd_slot_bytes(ctypes.byref(bad)) == 0
     h = ctypes.c_void_p()
     assert binding.lib.dd_create(ctypes.byref(bad), ctypes.byref(h)) == binding.DD_ERR_INVALID_ARG
     assert b"head_dim" in binding.lib.dd_last_error_message(None)
+
+
+def test_cluster_search_of_the_fused_selection_always_terminates():
+    """The search over cluster sizes with the device queries replaced by a callback: whatever the callback
+    answers, the search ends, and it returns 0 (two-kernel path) when nothing fits."""
+    from paper_2607_26475_b200 import build
+    build.build()
+    from paper_2607_26475_b200 import binding
+    ppc, smem = ctypes.c_int(), ctypes.c_size_t()
+
+    def pick(max_pages, problems, rows, allow16, answer):
+        calls = []
+
+        def fits(c, sm, _):
+            calls.append((c, sm))
+            assert len(calls) < 16, "the search does not terminate"
+            return 1 if answer(c, sm) else 0
+        cb = binding.PICK_FITS(fits)
+        got = binding.lib.dd_test_pick_cluster(max_pages, problems, 148, rows, 4, allow16, cb, None,
+                                                ctypes.byref(ppc), ctypes.byref(smem))
+        return got, calls
+
+    # config 2: 64 problems of 2048 pages -> 4 blocks each, 512 pages per block
+    got, calls = pick(2048, 64, 1, 1, lambda c, s: True)
+    assert got == 4 and ppc.value == 512 and smem.value == 512 * 4 * 4 + 2 * 2048 * 4
+    # one request of 64K pages: 16-block clusters when allowed, 8 otherwise
+    assert pick(65536, 8, 1, 1, lambda c, s: True)[0] == 16
+    assert pick(65536, 8, 1, 0, lambda c, s: True)[0] == 8
+    # 16 refused by the device: 8 is tried next, once
+    got, calls = pick(65536, 8, 1, 1, lambda c, s: c != 16)
+    assert got == 8 and [c for c, _ in calls] == [16, 8]
+    # the case that used to loop: 128K pages with four landmarks per page; 8 blocks exceed shared memory and
+    # the device refuses 16-block clusters
+    got, calls = pick(131072, 8, 4, 1, lambda c, s: False)
+    assert got == 0 and len(calls) <= 5
+    got, calls = pick(131072, 8, 1, 1, lambda c, s: False)
+    assert got == 0 and len(calls) <= 5
+    # nothing ever fits
+    assert pick(2048, 64, 1, 1, lambda c, s: False)[0] == 0
+    # a larger cluster is used when the preferred one does not fit
+    got, calls = pick(2048, 64, 1, 1, lambda c, s: c >= 8)
+    assert got == 8 and [c for c, _ in calls] == [4, 8]

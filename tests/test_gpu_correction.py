@@ -126,3 +126,46 @@ def test_corrected_chain_attends_the_true_sets(dd):
     # without correction the outputs are those of the predicted sets: they differ
     o3, _, _ = _run(dd, w, S, inp, depth=2, correct=False)
     assert np.abs(f32(o3) - f32(outs)).max() > 1e-3
+
+
+def test_corrected_chain_and_causal_tail_at_the_headline_request_shape(dd):
+    """The same two paths at the per-request shape of the batch-8 / 32K-context workload (2048 pages, 128
+    selected per KV head), not only at toy sizes: one request, two layers, two steps."""
+    S = 2
+    w = wl.small(wl.CONFIGS[2], n_layers=2, batch=1)
+    assert w.n_pages == 2048 and w.k_pages == 128
+    inp = _inputs(w, S)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    outs, merged, (missing, selected) = _run(dd, w, S, inp, depth=2, correct=True)
+    assert 0 < missing < selected
+    for t in range(S):
+        for l in range(w.n_layers):
+            _, sc = orc.select_topk(f32(q_steps[t, l][:, 0]), f32(lms[l]), npg.numpy(), w.k_pages)
+            for h in range(HKV):
+                check_selection(np.sort(merged[t, l, 0, h]), sc[0][h], w.k_pages, 0)
+            slot = orc.gather_kv(f32(store[l]), merged[t, l])
+            want, _ = orc.sparse_decode_attn(f32(q_steps[t, l]), slot, merged[t, l], ctx_len.numpy(), T)
+            check_attention(outs[t, l], want)
+    # causal tail through the pipelined call, same shape
+    g = torch.Generator().manual_seed(9)
+    k_new = torch.randn(S, w.n_layers, 1, 2, HKV, D, generator=g).to(torch.bfloat16)
+    v_new = torch.randn(S, w.n_layers, 1, 2, HKV, D, generator=g).to(torch.bfloat16)
+    c = dd.Context(n_layers=w.n_layers, batch=1, max_pages=w.n_pages, k_pages=w.k_pages)
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qd, kd, vd = q_steps.cuda(), k_new.cuda(), v_new.cuda()
+    o = torch.zeros_like(qd)
+    idxs = []
+    for t in range(S):
+        idxs.append([c.get_indices(t & 1, l).cpu().numpy() for l in range(w.n_layers)])
+        for l in range(w.n_layers):
+            c.decode_layer_step_causal(t, l, qd[t, l], kd[t, l], vd[t, l], o[t, l])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    c.close()
+    for t in range(S):
+        for l in range(w.n_layers):
+            slot = orc.gather_kv(f32(store[l]), idxs[t][l])
+            want, _ = orc.sparse_decode_attn_causal(f32(q_steps[t, l]), slot, idxs[t][l], ctx_len.numpy(), T,
+                                                    f32(k_new[t, l]), f32(v_new[t, l]))
+            check_attention(o[t, l], want)

@@ -1,4 +1,4 @@
-"""The allocation-free attention entry point against the context-based one.
+"""The allocation-free attention entry point against the context-based one and against the CPU oracle.
 
 Callers that may not allocate device memory (they run inside someone else's memory plan, or must not
 trigger the device synchronisation an allocation can cause) use dd_sparse_decode_attn_static, whose
@@ -11,7 +11,7 @@ import numpy as np
 import pytest
 import torch
 
-from tests._util import ATTN_MAX_ABS, ATTN_MEAN_ABS, f32
+from tests._util import ATTN_MAX_ABS, ATTN_MEAN_ABS, check_attention, f32
 
 pytestmark = pytest.mark.gpu
 
@@ -40,6 +40,11 @@ def _case(dd, seed, B, P, k, splits_ctx, splits_static, ctx_len):
     err = np.abs(f32(got).astype(np.float64) - f32(want).astype(np.float64))
     assert err.max() <= ATTN_MAX_ABS and err.mean() <= ATTN_MEAN_ABS, (err.max(), err.mean())
     np.testing.assert_allclose(got_lse.cpu().numpy(), want_lse.cpu().numpy(), atol=2e-3, rtol=1e-4)
+    # and directly against the oracle, on the slot the caller handed in
+    from oracle import dd_oracle as orc
+    ref, ref_lse = orc.sparse_decode_attn(f32(q), f32(slot), idx.cpu().numpy(), np.asarray(ctx_len), T)
+    check_attention(got, ref)
+    np.testing.assert_allclose(got_lse.cpu().numpy(), ref_lse, atol=2e-3, rtol=1e-4)
     return err.max()
 
 
@@ -67,3 +72,34 @@ def test_static_entry_point_rejects_what_does_not_fit():
     with pytest.raises(dd.DDError) as e:
         dd.sparse_decode_attn_static(q, slot, idx, cl, q.clone(), n_splits=k + 1)
     assert e.value.code == dd.DD_ERR_INVALID_ARG
+
+
+def test_static_entry_point_rejects_memory_the_device_cannot_use():
+    """Pageable host memory (or a misaligned pointer) for any tensor is an error code before anything is
+    enqueued, never a device fault: the checks run on the host and launch nothing."""
+    from paper_2607_26475_b200 import binding as dd
+    B, k = 2, 16
+    q = torch.zeros((B, 2, 32, D), dtype=torch.bfloat16, device="cuda")
+    idx = torch.arange(k, dtype=torch.int32).repeat(B, HKV, 1).contiguous().cuda()
+    cl = torch.full((B,), k * T, dtype=torch.int32, device="cuda")
+    slot = torch.zeros((B, HKV, 2, k * T, D), dtype=torch.bfloat16, device="cuda")
+    out = torch.full_like(q, 7.0)
+    good = dict(q=q, slot=slot, idx=idx, ctx_len=cl, out=out)
+    for name in ("q", "slot", "idx", "ctx_len", "out"):
+        args = dict(good)
+        args[name] = good[name].cpu()                                    # pageable host memory
+        with pytest.raises(dd.DDError) as e:
+            dd.sparse_decode_attn_static(args["q"], args["slot"], args["idx"], args["ctx_len"], args["out"], n_splits=2)
+        assert e.value.code == dd.DD_ERR_INVALID_ARG and name in str(e.value)
+    with pytest.raises(dd.DDError) as e:
+        dd.sparse_decode_attn_static(q, slot, idx, cl, out, torch.zeros((B, 2, 32), dtype=torch.float32), n_splits=2)
+    assert e.value.code == dd.DD_ERR_INVALID_ARG and "out_lse" in str(e.value)
+    with pytest.raises(dd.DDError) as e:                                 # bf16 tensors must be 16-byte aligned
+        q_off = torch.zeros(q.numel() + 8, dtype=torch.bfloat16, device="cuda")[1:1 + q.numel()].view(q.shape)
+        dd.sparse_decode_attn_static(q_off, slot, idx, cl, out, n_splits=2)
+    assert e.value.code == dd.DD_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())                                      # nothing ran
+    dd.sparse_decode_attn_static(q, slot, idx, cl, out, n_splits=2)      # the device is still usable
+    torch.cuda.synchronize()
+    assert bool((out == 0.0).all())
