@@ -31,3 +31,12 @@ def throughput(ms_local: float, tokens_local: int, device="cpu") -> float:
 def host_budget_per_rank(available_bytes: int, local_world: int, fraction: float = 0.6) -> int:
     """Pinned host memory one rank may use for its store share."""
     return int(available_bytes * fraction / max(1, local_world))
+
+
+def gather_per_rank(value: float) -> list[float]:
+    """The same scalar from every rank, in rank order (on every rank); [value] without a process group."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(value)]
+    out = [None] * dist.get_world_size()
+    dist.all_gather_object(out, float(value))
+    return [float(v) for v in out]
