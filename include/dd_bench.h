@@ -73,12 +73,15 @@ int dd_set_bulk_wait(dd_ctx* ctx, double wait_seconds, int inflate_first_stage);
 
 /* The cluster-size search of the fused selection kernel with the device queries replaced by a callback, so that
  * it can be tested without a GPU: returns the chosen blocks per (request, KV head), or 0 when no cluster size
- * fits (the two-kernel path is then used). fits(blocks, shared_bytes, user) says whether clusters of that many
- * blocks with that much dynamic shared memory per block can be resident; allow16 says whether 16-block
- * (non-portable) clusters may be tried. rows_per_page = landmarks per page, group = query heads per KV head. */
+ * fits (the two-kernel path is then used). fits(blocks, shared_bytes, user) returns how many clusters of that many
+ * blocks with that much dynamic shared memory per block the device holds at once (0 = cannot run); a size whose
+ * clusters are all resident (fits >= problems) is preferred. allow16 says whether 16-block
+ * (non-portable) clusters may be tried. rows_per_page = landmarks per page, group = query heads per KV head;
+ * ring_stages receives the depth of the scoring phase's shared-memory ring (tiles per warp), logits_global
+ * whether the logits go to global scratch instead of shared memory. */
 int dd_test_pick_cluster(int max_pages, int problems, int sm_count, int rows_per_page, int group, int allow16,
                          int (*fits)(int blocks, size_t shared_bytes, void* user), void* user, int* pages_per_block,
-                         size_t* shared_bytes);
+                         size_t* shared_bytes, int* ring_stages, int* logits_global);
 
 #ifdef __cplusplus
 }

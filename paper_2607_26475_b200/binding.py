@@ -113,7 +113,7 @@ def _load() -> C.CDLL:
     lib.dd_last_device_error.argtypes = [vp, C.POINTER(ip), C.POINTER(ip)]
     lib.dd_gather_stats.argtypes = [vp, C.POINTER(C.c_ulonglong), ip]
     lib.dd_set_bulk_wait.argtypes = [vp, C.c_double, ip]
-    lib.dd_test_pick_cluster.argtypes = [ip, ip, ip, ip, ip, ip, PICK_FITS, vp, C.POINTER(ip), C.POINTER(C.c_size_t)]
+    lib.dd_test_pick_cluster.argtypes = [ip, ip, ip, ip, ip, ip, PICK_FITS, vp, C.POINTER(ip), C.POINTER(C.c_size_t), C.POINTER(ip), C.POINTER(ip)]
     lib.dd_static_scratch_capacity.argtypes = []
     lib.dd_static_scratch_capacity.restype = C.c_size_t
     lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7

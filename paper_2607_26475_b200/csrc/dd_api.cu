@@ -120,7 +120,8 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
   dd_sizes z;
   const size_t B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads, P = c->max_pages;
   const size_t G = Hq / Hkv, tiles = (P + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
-  z.score_s = up256(B * Hkv * P * G * 4);
+  const size_t Rr = c->landmark_chunk_tokens ? DD_T / c->landmark_chunk_tokens : 1;
+  z.score_s = up256(2 * B * Hkv * P * Rr * G * 4);
   z.score_part = up256(B * Hq * tiles * 8);
   z.topk_keys = up256(B * Hkv * P * 4);
   z.part_o = up256(B * Hkv * (size_t)S * 8 * DD_D * 4);

@@ -31,9 +31,11 @@ struct dd_ctx {
   int sel_cluster;       // blocks per cluster of the fused selection kernel; 0 = two-kernel path
   int sel_ppc;           // pages per block of the fused selection
   int sel_smem_bytes;
+  int sel_stages;        // tiles per warp in the scoring ring of the fused selection
+  int sel_logits_global; // 1: the fused selection keeps its logits in score_s (two buffers) instead of shared memory
   size_t slot_bytes;
   // scratch (device)
-  float* score_s;        // [B][Hkv][P][G] scaled logits
+  float* score_s;        // [2][B][Hkv][P*R][G] scaled logits (second buffer: selections on the selection stream)
   float2* score_part;    // [B][Hq][score_tiles] per-tile (max, sum exp)
   uint32_t* topk_keys;   // [B][Hkv][P] order-preserving keys when a request does not fit shared memory
   float* attn_part_o;    // [B][Hkv][S][8][128] unnormalised partial outputs

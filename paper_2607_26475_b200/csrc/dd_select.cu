@@ -345,21 +345,31 @@ __global__ void __launch_bounds__(TOPK_THREADS) dd_topk_kernel(
 // Fused selection: one thread-block cluster per (request, KV head).
 //
 // Block `rank` of the cluster scores the pages [rank*ppc, (rank+1)*ppc) and keeps their logits in its own
-// shared memory; what the blocks must agree on travels through distributed shared memory:
-//   1. per-head (max, sum exp) of every block      -> log-sum-exp of the request
-//   2. min / max of the order-preserving keys      -> digit positions of the radix select
-//   3. per radix pass, the sums of 8-bin groups and the 8 bins of one group; then the few keys that share
-//      the leading digits                          -> the k-th largest key (every block derives it)
-//   4. per-block counts of selected pages          -> where each block's pages go in the ascending output
+// shared memory; what the blocks must agree on is published in shared memory and read by the peers through
+// distributed shared memory after a cluster barrier:
+//   barrier 1   per-head (max, sum exp, min) of every block's logits  -> log-sum-exp of the request and a range
+//               [lo, hi] that certainly holds every key (key = max over heads of logit - lse, so
+//               max_h(min_h - lse_h) <= key <= max_h(max_h - lse_h)): no separate min / max exchange
+//   barrier 2   per radix pass (11-bit digits cut from the top of key - lo), the sums of 8-bin groups; the 8 bins
+//               of the group where the count crosses k are then read directly
+//   barrier 3   the few keys that share the leading digits with the k-th largest, and how many local keys lie
+//               above them -> every block ranks the candidates (the k-th largest key) and derives every other
+//               block's contribution, i.e. its own output offset, without a further exchange
+//   barrier 4   nobody leaves while a peer may still read its shared memory (arrive after the last remote read,
+//               wait at the very end)
 // Nothing but the landmarks is read from global memory, and nothing but the index set is written.
 // ------------------------------------------------------------------------------------------------
 namespace cg = cooperative_groups;
 
-
 constexpr int SEL_THREADS = 256;
 constexpr int SEL_WARPS = SEL_THREADS / 32;
-constexpr int SEL_CAND_MAX = 512;          // keys sharing a radix prefix that are ranked directly
+constexpr int SEL_CAND_MAX = 256;          // keys sharing a radix prefix that are ranked directly
 constexpr int SEL_MAX_SMEM = 200 * 1024;   // dynamic shared memory the fused kernel may be launched with
+constexpr int SEL_MAX_CLUSTER = 16;
+
+__device__ __forceinline__ void dd_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void dd_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void dd_cluster_sync() { dd_cluster_arrive(); dd_cluster_wait(); }
 
 // Exclusive prefix sum over the 256 threads of the block; `total` is returned to every thread.
 __device__ __forceinline__ unsigned dd_scan256_excl(unsigned v, unsigned* warp_tot, unsigned& total) {
@@ -385,24 +395,69 @@ __device__ __forceinline__ unsigned dd_scan256_excl(unsigned v, unsigned* warp_t
   return wexcl + inc - v;
 }
 
+// What a block publishes for its peers.
+struct dd_sel_pub {
+  float m[8], l[8];            // per head of the group: reference and sum of exp(s - reference) over this block's logits
+  float mn[8], mx[8];          // smallest and largest logit
+  unsigned above;              // local pages certainly selected: forced ones and keys above the candidates' digits
+  unsigned eq;                 // local keys equal to the threshold when the digits resolve it exactly
+  unsigned cand_n;             // local candidate keys listed in cand[]
+  uint32_t cand[SEL_CAND_MAX];
+};
+
+// 16-byte asynchronous copy global -> shared memory (bypasses registers and L1), and its group bookkeeping.
+__device__ __forceinline__ void dd_cp_async16(void* smem, const void* gmem) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void dd_cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void dd_cp_async_wait_pending(int n) {   // at most n groups still in flight (n <= 3)
+  if (n >= 3) asm volatile("cp.async.wait_group 3;" ::: "memory");
+  else if (n == 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+  else if (n == 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+  else asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+// Fragments of one 16-row tile of landmarks: rows gl and gl + 8, channels [32kk + 8t, +8) for kk = 0..3.
+struct dd_sel_frag {
+  uint4 lo[4], hi[4];
+};
+
+__device__ __forceinline__ void dd_sel_load_tile(dd_sel_frag& f, const __nv_bfloat16* lm_bg, int row0, int row_max, int gl,
+                                                 int t) {
+  const int pa = min(row0 + gl, row_max);                 // stay inside the tensor; rows past the end are discarded later
+  const int pb = min(row0 + gl + 8, row_max);
+  const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D);
+  const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D);
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    f.lo[kk] = dd_ld_stream(ra + kk * 4 + t);
+    f.hi[kk] = dd_ld_stream(rb + kk * 4 + t);
+  }
+}
+
 __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     const __nv_bfloat16* __restrict__ q, int q_req_stride, int q_token_off, const __nv_bfloat16* __restrict__ lm,
     const int* __restrict__ n_pages, int* __restrict__ out_idx, float* __restrict__ out_scores, int P, int G, int Hkv,
-    int k, int forced, int ppc, int* err_word, int R, const int* __restrict__ ctx_len) {
+    int k, int forced, int ppc, int* err_word, int R, const int* __restrict__ ctx_len, int ring_stages, float* __restrict__ s_glob) {
   extern __shared__ __align__(16) unsigned char sel_smem[];
-  float* s_sm = reinterpret_cast<float*>(sel_smem);                    // [ppc * R][G] logits; a page's key in its first slot
-  unsigned* hist = reinterpret_cast<unsigned*>(sel_smem + (size_t)ppc * R * G * 4);   // [2][RADIX_BINS]
-  const int KS = R * G;                                                // floats per page
-  __shared__ float2 cta_ml[8];
-  __shared__ unsigned cta_minmax[2];
-  __shared__ unsigned cta_cnt[2];
-  __shared__ float2 red[SEL_WARPS][8];
-  __shared__ float lse_s[8];
-  __shared__ unsigned warp_tot[SEL_WARPS];
-  __shared__ unsigned sh_bin, sh_above, sh_grp, sh_cnt, sh_thr, cand_n;
+  // logits [ppc * R][G] of this block's rows: in shared memory when they leave room for a deep ring, otherwise in
+  // the context's global scratch (written and re-read by this block only; it stays in L2)
+  float* s_sm = s_glob ? s_glob + ((size_t)(blockIdx.z * Hkv + blockIdx.y) * P + (size_t)blockIdx.x * ppc) * R * G
+                       : reinterpret_cast<float*>(sel_smem);
+  // the landmark ring of the scoring phase shares its memory with the keys and histograms of the later phases
+  uint4* ring = reinterpret_cast<uint4*>(sel_smem + (s_glob ? 0 : (size_t)ppc * R * G * 4));   // [warp][stage][8][32] x 16 B
+  uint32_t* keys = reinterpret_cast<uint32_t*>(ring);                                   // [ppc] key of every local page
+  unsigned* hist = reinterpret_cast<unsigned*>(keys + ppc);                             // [2][RADIX_BINS]
+  __shared__ dd_sel_pub pub;
   __shared__ unsigned grp[2][SEL_THREADS];
+  __shared__ float red_m[SEL_WARPS][8], red_l[SEL_WARPS][8], red_mn[SEL_WARPS][8], red_mx[SEL_WARPS][8];
+  __shared__ float pull_m[SEL_MAX_CLUSTER][8], pull_l[SEL_MAX_CLUSTER][8], pull_mn[SEL_MAX_CLUSTER][8], pull_mx[SEL_MAX_CLUSTER][8];
+  __shared__ float lse_s[8], lo_s[8], hi_s[8];
+  __shared__ unsigned warp_tot[SEL_WARPS];
+  __shared__ unsigned warp_gt[SEL_WARPS], warp_eq[SEL_WARPS];
+  __shared__ unsigned sh_above, sh_grp, sh_thr, sh_base_gt, sh_base_eq;
   __shared__ unsigned cnt8[8];
-  __shared__ uint32_t cand[SEL_CAND_MAX];
+  __shared__ unsigned peer_above[SEL_MAX_CLUSTER], peer_eq[SEL_MAX_CLUSTER], peer_cand[SEL_MAX_CLUSTER];
   __shared__ uint32_t all_c[SEL_CAND_MAX];
 
   cg::cluster_group cl = cg::this_cluster();
@@ -427,11 +482,15 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   int n_rows_req = np * R;
   if (R > 1) n_rows_req = min(n_rows_req, (ctx_len[b] + DD_T / R - 1) / (DD_T / R));
   const int n_local_rows = max(0, min(n_rows_req, (p_lo + ppc) * R) - p_lo * R);
-  if (tid == 0) { cta_minmax[0] = 0xFFFFFFFFu; cta_minmax[1] = 0u; cta_cnt[0] = 0u; cta_cnt[1] = 0u; cand_n = 0u; }
+  if (tid == 0) { pub.above = 0u; pub.eq = 0u; pub.cand_n = 0u; sh_base_gt = 0u; sh_base_eq = 0u; }
 
-  // ---- A. logits of this block's pages (same MMA formulation as dd_score_kernel), kept in shared memory
-  float m_run[2] = {-INFINITY, -INFINITY};
+  // ---- A. logits of this block's rows, kept in shared memory. 16 landmarks are the M rows of a bf16 MMA, the G heads
+  // its N columns (same fragment trick as dd_score_kernel). Every lane copies the fragments it will use itself with
+  // 16-byte asynchronous copies into a private ring in shared memory (ring_stages tiles deep per warp), so that
+  // several tiles per warp are in flight whatever the register allocation; no lane reads another lane's bytes.
+  float m_run[2] = {-INFINITY, -INFINITY};       // heads 2t, 2t+1: reference of the running sum
   float l_run[2] = {0.f, 0.f};
+  float mn_run[2] = {INFINITY, INFINITY}, mx_run[2] = {-INFINITY, -INFINITY};   // smallest and largest logit
   {
     uint4 qf[4];
     if (gl < G) {
@@ -446,47 +505,73 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * R * DD_D;
     const float scale = rsqrtf((float)DD_D);
     const int row_lo = p_lo * R, row_max = P * R - 1;
-    for (int t0 = warp * 32; t0 < n_local_rows; t0 += SEL_WARPS * 32) {  // two 16-row MMA tiles per trip
-      uint4 lo[2][4], hi[2][4];
+    const int n_tiles = (n_local_rows + 15) >> 4;
+    auto consume = [&](const dd_sel_frag& f, int tile) {
+      // two independent accumulator chains halve the latency of the dependent MMAs
+      float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        const int pa = min(row_lo + t0 + mt * 16 + gl, row_max);       // stay inside the tensor; discarded later
-        const int pb = min(row_lo + t0 + mt * 16 + gl + 8, row_max);
-        const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D);
-        const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D);
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          lo[mt][kk] = dd_ld_stream(ra + kk * 4 + t);
-          hi[mt][kk] = dd_ld_stream(rb + kk * 4 + t);
-        }
+      for (int kk = 0; kk < 4; ++kk) {
+        dd_mma_bf16(acc, f.lo[kk].x, f.hi[kk].x, f.lo[kk].y, f.hi[kk].y, qf[kk].x, qf[kk].y);
+        dd_mma_bf16(acc2, f.lo[kk].z, f.hi[kk].z, f.lo[kk].w, f.hi[kk].w, qf[kk].z, qf[kk].w);
       }
+      // acc[0], acc[1]: row gl, heads 2t, 2t+1; acc[2], acc[3]: row gl + 8
+      const int r0 = tile * 16 + gl, r1 = r0 + 8;
+      const bool ok0 = r0 < n_local_rows, ok1 = r1 < n_local_rows;
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
-          dd_mma_bf16(acc, lo[mt][kk].x, hi[mt][kk].x, lo[mt][kk].y, hi[mt][kk].y, qf[kk].x, qf[kk].y);
-          dd_mma_bf16(acc, lo[mt][kk].z, hi[mt][kk].z, lo[mt][kk].w, hi[mt][kk].w, qf[kk].z, qf[kk].w);
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const int pl = t0 + mt * 16 + gl + r * 8;                     // landmark row within the block
-          if (pl < n_local_rows) {
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              const int h = 2 * t + c;
-              if (h < G) {
-                const float v = acc[2 * r + c] * scale;
-                s_sm[(size_t)pl * G + h] = v;
-                const float mn = fmaxf(m_run[c], v);
-                l_run[c] = l_run[c] * expf(m_run[c] - mn) + expf(v - mn);
-                m_run[c] = mn;
-              }
-            }
+      for (int c = 0; c < 2; ++c) {
+        const int h = 2 * t + c;
+        if (h < G && ok0) {
+          const float v0 = (acc[c] + acc2[c]) * scale;
+          const float v1 = ok1 ? (acc[2 + c] + acc2[2 + c]) * scale : v0;
+          s_sm[(size_t)r0 * G + h] = v0;
+          if (ok1) s_sm[(size_t)r1 * G + h] = v1;
+          const float vmax = fmaxf(v0, v1);
+          mx_run[c] = fmaxf(mx_run[c], vmax);
+          mn_run[c] = fminf(mn_run[c], fminf(v0, v1));
+          // running sum of exp(v - m_run): the reference m_run moves only when a value exceeds it by a wide margin
+          // (any reference gives the same log-sum-exp as long as nothing overflows)
+          if (vmax > m_run[c] + 40.f) {
+            l_run[c] *= __expf(m_run[c] - vmax);
+            m_run[c] = vmax;
           }
+          l_run[c] += __expf(v0 - m_run[c]) + (ok1 ? __expf(v1 - m_run[c]) : 0.f);
         }
       }
+    };
+    uint4* my_ring = ring + (size_t)warp * ring_stages * 256 + lane;   // [stage][8][32] of this warp, this lane's column
+    auto issue = [&](int tile, int slot) {                 // always commits a group, possibly an empty one
+      if (tile < n_tiles) {
+        const int pa = min(row_lo + tile * 16 + gl, row_max);   // stay inside the tensor; rows past the end are discarded
+        const int pb = min(row_lo + tile * 16 + gl + 8, row_max);
+        const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D) + t;
+        const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D) + t;
+        uint4* dst = my_ring + slot * 256;
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          dd_cp_async16(dst + kk * 32, ra + kk * 4);
+          dd_cp_async16(dst + (4 + kk) * 32, rb + kk * 4);
+        }
+      }
+      dd_cp_async_commit();
+    };
+    const int ahead = ring_stages - 1;                     // tiles in flight per warp
+    for (int s = 0; s < ahead; ++s) issue(warp + s * SEL_WARPS, s);
+    int slot = 0, slot_issue = ahead;
+    for (int tile = warp; tile < n_tiles; tile += SEL_WARPS) {
+      issue(tile + ahead * SEL_WARPS, slot_issue);
+      dd_cp_async_wait_pending(ahead);                     // the oldest group, this tile, has landed
+      dd_sel_frag f;
+      const uint4* src = my_ring + slot * 256;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        f.lo[kk] = src[kk * 32];
+        f.hi[kk] = src[(4 + kk) * 32];
+      }
+      consume(f, tile);
+      slot = slot + 1 == ring_stages ? 0 : slot + 1;
+      slot_issue = slot_issue + 1 == ring_stages ? 0 : slot_issue + 1;
     }
+    dd_cp_async_wait_pending(0);
   }
 #pragma unroll
   for (int c = 0; c < 2; ++c) {
@@ -495,89 +580,120 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       const float m2 = __shfl_xor_sync(0xffffffffu, m_run[c], off);
       const float l2 = __shfl_xor_sync(0xffffffffu, l_run[c], off);
       dd_ml_merge(m_run[c], l_run[c], m2, l2, false);
+      mn_run[c] = fminf(mn_run[c], __shfl_xor_sync(0xffffffffu, mn_run[c], off));
+      mx_run[c] = fmaxf(mx_run[c], __shfl_xor_sync(0xffffffffu, mx_run[c], off));
     }
   }
   if (gl == 0) {
-    red[warp][2 * t] = make_float2(m_run[0], l_run[0]);
-    red[warp][2 * t + 1] = make_float2(m_run[1], l_run[1]);
-  }
-  __syncthreads();
-  if (tid < 8) {
-    float m = red[0][tid].x, l = red[0][tid].y;
 #pragma unroll
-    for (int w = 1; w < SEL_WARPS; ++w) dd_ml_merge(m, l, red[w][tid].x, red[w][tid].y, false);
-    cta_ml[tid] = make_float2(m, l);
-  }
-  // ---- B. log-sum-exp of the whole request: every block merges the partials of all blocks
-  cl.sync();
-  if (tid < G) {
-    float m = -INFINITY, l = 0.f;
-    for (int r = 0; r < C; ++r) {
-      const float2 v = *cl.map_shared_rank(&cta_ml[tid], r);
-      dd_ml_merge(m, l, v.x, v.y, false);
+    for (int c = 0; c < 2; ++c) {
+      red_m[warp][2 * t + c] = m_run[c];
+      red_l[warp][2 * t + c] = l_run[c];
+      red_mn[warp][2 * t + c] = mn_run[c];
+      red_mx[warp][2 * t + c] = mx_run[c];
     }
-    lse_s[tid] = m + logf(l);
+  }
+  __syncthreads();                               // every warp is done with its ring: the memory becomes keys + histograms
+  for (int i = tid; i < 2 * RADIX_BINS; i += SEL_THREADS) hist[i] = 0u;
+  if (tid < 8) {
+    float m = red_m[0][tid], l = red_l[0][tid], mn = red_mn[0][tid], mx = red_mx[0][tid];
+#pragma unroll
+    for (int w = 1; w < SEL_WARPS; ++w) {
+      dd_ml_merge(m, l, red_m[w][tid], red_l[w][tid], false);
+      mn = fminf(mn, red_mn[w][tid]);
+      mx = fmaxf(mx, red_mx[w][tid]);
+    }
+    pub.m[tid] = m;
+    pub.l[tid] = l;
+    pub.mn[tid] = mn;
+    pub.mx[tid] = mx;
+  }
+  // ---- B. log-sum-exp of the whole request and the key range, from every block's partials
+  dd_cluster_sync();
+  if (tid < C * 8) {                             // one thread per (peer, head): all remote reads are in flight at once
+    const int r = tid >> 3, h = tid & 7;
+    const dd_sel_pub* pr = cl.map_shared_rank(&pub, r);
+    pull_m[r][h] = pr->m[h];
+    pull_l[r][h] = pr->l[h];
+    pull_mn[r][h] = pr->mn[h];
+    pull_mx[r][h] = pr->mx[h];
   }
   __syncthreads();
-
-  // ---- C. keys in place of the first logit of every page; block min / max of the non-forced keys
+  if (tid < G) {
+    float m = -INFINITY, l = 0.f, mn = INFINITY, mx = -INFINITY;
+    for (int r = 0; r < C; ++r) {
+      dd_ml_merge(m, l, pull_m[r][tid], pull_l[r][tid], false);
+      mn = fminf(mn, pull_mn[r][tid]);
+      mx = fmaxf(mx, pull_mx[r][tid]);
+    }
+    const float lse = m + logf(l);
+    lse_s[tid] = lse;
+    lo_s[tid] = mn - lse;
+    hi_s[tid] = mx - lse;
+  }
+  __syncthreads();
+  // ---- C. keys: group maximum of the log-probabilities (a page takes the best of its existing chunks) in
+  // order-preserving integer form, and the first histogram over the leading digits of key - lo
+  uint32_t klo, khi;
+  {
+    float lo = -INFINITY, hi = -INFINITY;
+    for (int h = 0; h < G; ++h) { lo = fmaxf(lo, lo_s[h]); hi = fmaxf(hi, hi_s[h]); }
+    klo = dd_orderable(lo);
+    khi = dd_orderable(hi);
+  }
+  const int n_free_local = max(0, min(n_free, p_lo + ppc) - p_lo);     // local pages that take part in the select
+  const int nbits = khi > klo ? 32 - __clz(khi - klo) : 0;
+  int hi_bits = nbits;                           // bits of (key - lo) not resolved yet; digits are cut from the top
   {
     float lse[8];
 #pragma unroll
     for (int h = 0; h < 8; ++h) lse[h] = h < G ? lse_s[h] : 0.f;
-    uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+    const int width = hi_bits < RADIX_BITS ? hi_bits : RADIX_BITS;
+    const int shift = hi_bits - width;
+    const bool quad = G == 4 && R == 1;          // the common shape: one 16-byte read per page
     for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
       float c = -INFINITY;
-      for (int r = 0; r < R; ++r) {              // a page takes the best of its existing chunks
-        if (pl * R + r < n_local_rows) {
+      if (quad) {
+        const float4 v = *reinterpret_cast<const float4*>(s_sm + (size_t)pl * 4);
+        c = fmaxf(fmaxf(v.x - lse[0], v.y - lse[1]), fmaxf(v.z - lse[2], v.w - lse[3]));
+      } else {
+        for (int r = 0; r < R; ++r) {
+          if (pl * R + r < n_local_rows) {
 #pragma unroll
-          for (int h = 0; h < 8; ++h)
-            if (h < G) c = fmaxf(c, s_sm[((size_t)pl * R + r) * G + h] - lse[h]);
+            for (int h = 0; h < 8; ++h)
+              if (h < G) c = fmaxf(c, s_sm[((size_t)pl * R + r) * G + h] - lse[h]);
+          }
         }
       }
       const int p = p_lo + pl;
       if (out_scores) out_scores[bg * P + p] = expf(c);
       uint32_t key = dd_orderable(c);
+      key = key < klo ? klo : (key > khi ? khi : key);                  // the range holds every key; keep the digits safe
       if (p >= n_free) key = 0xFFFFFFFFu;
-      else { kmin = min(kmin, key); kmax = max(kmax, key); }
-      reinterpret_cast<uint32_t*>(s_sm)[(size_t)pl * KS] = key;
+      else if (width > 0) atomicAdd(&hist[(key - klo) >> shift], 1u);
+      keys[pl] = key;
     }
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { atomicMin(&cta_minmax[0], kmin); atomicMax(&cta_minmax[1], kmax); }
   }
-  const uint32_t* keys = reinterpret_cast<const uint32_t*>(s_sm);      // key of local page pl at keys[pl * KS]
-  cl.sync();
-  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
-  for (int r = 0; r < C; ++r) {
-    kmin = min(kmin, *cl.map_shared_rank(&cta_minmax[0], r));
-    kmax = max(kmax, *cl.map_shared_rank(&cta_minmax[1], r));
-  }
-  const int n_free_local = max(0, min(n_free, p_lo + ppc) - p_lo);     // local pages that take part in the select
 
-  // ---- D. the k_free-th largest key. MSB-first radix passes on (key - min); a pass exchanges only the sums
-  // of 8-bin groups and then the 8 bins of the group where the count crosses k. As soon as the crossing bin
-  // holds few keys, those keys themselves are exchanged and ranked, which ends the search.
-  uint32_t thr = 0xFFFFFFFFu;
-  unsigned k_rem = 0;
+  // ---- D. the k_free-th largest key. MSB-first radix passes on (key - lo); a pass exchanges only the sums of 8-bin
+  // groups and reads the 8 bins of the group where the count crosses k. It ends when the digits are exhausted or
+  // the crossing bin holds few keys.
+  unsigned long long prefix = 0;
+  unsigned k_rem = (unsigned)k_free;
+  int shift = hi_bits;                           // bits below the resolved prefix
   if (k_free > 0) {
-    const uint32_t range = kmax - kmin;
-    const int nbits = 32 - __clz(range);
-    unsigned long long prefix = 0;
-    k_rem = (unsigned)k_free;
-    thr = kmin;                                   // all keys equal (nbits == 0): take the first k_free of them
-    bool done = false;
-    int hi = nbits;                               // bits of (key - min) not resolved yet; digits are cut from the top
-    for (int pass = 0; hi > 0 && !done; ++pass) {
-      const int width = hi < RADIX_BITS ? hi : RADIX_BITS;
-      const int shift = hi - width;
+    for (int pass = 0; shift > 0; ++pass) {
+      const int width = shift < RADIX_BITS ? shift : RADIX_BITS;
+      const int nshift = shift - width;
       unsigned* h = hist + (pass & 1) * RADIX_BINS;                     // double-buffered: peers may still read the other
       unsigned* gp = grp[pass & 1];
-      for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) h[i] = 0u;
-      __syncthreads();
-      for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
-        const unsigned long long rel = (unsigned long long)(keys[(size_t)pl * KS] - kmin);
-        if ((rel >> hi) == prefix) atomicAdd(&h[(unsigned)(rel >> shift) & ((1u << width) - 1u)], 1u);
+      if (pass > 0) {
+        for (int i = tid; i < RADIX_BINS; i += SEL_THREADS) h[i] = 0u;
+        __syncthreads();
+        for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
+          const unsigned long long rel = (unsigned long long)(keys[pl] - klo);
+          if ((rel >> shift) == prefix) atomicAdd(&h[(unsigned)(rel >> nshift) & ((1u << width) - 1u)], 1u);
+        }
       }
       __syncthreads();
       {                                           // thread i owns the 8 bins [2047-8i-7, 2047-8i]
@@ -586,7 +702,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
         for (int jb = 0; jb < 8; ++jb) sum8 += h[RADIX_BINS - 1 - 8 * tid - jb];
         gp[tid] = sum8;
       }
-      cl.sync();
+      dd_cluster_sync();
       unsigned tot = 0;
       for (int r = 0; r < C; ++r) tot += cl.map_shared_rank(gp, r)[tid];
       unsigned total;
@@ -600,94 +716,157 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
         cnt8[tid] = c8;
       }
       __syncthreads();
-      if (tid == 0) {
-        unsigned ab = sh_above;
-        for (int jb = 0; jb < 8; ++jb) {
-          if (ab < k_rem && k_rem <= ab + cnt8[jb]) { sh_bin = RADIX_BINS - 1 - 8 * gsel - jb; sh_above = ab; sh_cnt = cnt8[jb]; break; }
-          ab += cnt8[jb];
-        }
+      unsigned ab = sh_above, bin = 0, bin_cnt = 0;  // every thread walks the 8 bins itself
+#pragma unroll
+      for (int jb = 0; jb < 8; ++jb) {
+        const unsigned c8 = cnt8[jb];
+        if (bin_cnt == 0 && ab < k_rem && k_rem <= ab + c8) { bin = RADIX_BINS - 1 - 8 * gsel - jb; bin_cnt = c8; }
+        if (bin_cnt == 0) ab += c8;
       }
-      __syncthreads();
-      prefix = (prefix << width) | sh_bin;
-      k_rem -= sh_above;                          // keys in higher bins are all selected
-      const unsigned bin_cnt = sh_cnt;
-      hi = shift;
-      __syncthreads();
-      if (hi == 0) {
-        thr = kmin + (uint32_t)prefix;            // k_rem of the keys equal to thr are still to be taken
-      } else if (bin_cnt <= (unsigned)SEL_CAND_MAX) {
-        // few keys share the prefix: every block lists its own, all blocks read all lists and rank them
-        for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
-          const uint32_t key = keys[(size_t)pl * KS];
-          if (((unsigned long long)(key - kmin) >> shift) == prefix) cand[atomicAdd(&cand_n, 1u)] = key;
-        }
-        cl.sync();
-        unsigned off = 0;
-        for (int r = 0; r < C; ++r) {
-          const unsigned n_r = *cl.map_shared_rank(&cand_n, r);
-          const uint32_t* cr = cl.map_shared_rank(cand, r);
-          for (unsigned i = tid; i < n_r; i += SEL_THREADS) all_c[off + i] = cr[i];
-          off += n_r;
-        }
-        __syncthreads();
-        for (unsigned i = tid; i < off; i += SEL_THREADS) {
-          const uint32_t v = all_c[i];
-          unsigned gtc = 0, gec = 0;
-          for (unsigned j = 0; j < off; ++j) {
-            const uint32_t u = all_c[j];
-            gtc += u > v;
-            gec += u >= v;
-          }
-          if (gtc < k_rem && k_rem <= gec) { sh_thr = v; sh_above = gtc; }   // equal candidates write equal values
-        }
-        __syncthreads();
-        thr = sh_thr;
-        k_rem -= sh_above;
-        done = true;
-      }
+      prefix = (prefix << width) | bin;
+      k_rem -= ab;                                // keys in higher bins are all selected
+      shift = nshift;
+      __syncthreads();                            // sh_grp, sh_above and cnt8 are rewritten by the next pass
+      if (bin_cnt <= (unsigned)SEL_CAND_MAX) break;
     }
   }
 
-  // ---- E. how many pages each block contributes, then ordered compaction of this block's pages
+  // ---- E. publish what the peers need to finish: how many local pages are certainly selected, and the local keys
+  // that share the prefix (listed when digits remain, only counted when the prefix is the whole key)
   {
-    unsigned gt = 0, eq = 0;
-    for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
-      const uint32_t key = keys[(size_t)pl * KS];
-      if (p_lo + pl >= n_free || key > thr) ++gt;
-      else if (key == thr) ++eq;
+    unsigned n_above = 0, n_eq = 0;
+    for (int base = warp * 32; base < n_local; base += SEL_THREADS) {
+      const int pl = base + lane;
+      bool ab = false, eq = false;
+      uint32_t key = 0;
+      if (pl < n_local) {
+        key = keys[pl];
+        if (p_lo + pl >= n_free) ab = true;
+        else if (k_free > 0) {
+          const unsigned long long dg = (unsigned long long)(key - klo) >> shift;
+          ab = dg > prefix;
+          eq = dg == prefix;
+        }
+      }
+      n_above += __popc(__ballot_sync(0xffffffffu, ab));
+      if (shift > 0) {
+        const unsigned be = __ballot_sync(0xffffffffu, eq);
+        unsigned base_slot = 0;
+        if (lane == 0 && be) base_slot = atomicAdd(&pub.cand_n, (unsigned)__popc(be));
+        base_slot = __shfl_sync(0xffffffffu, base_slot, 0);
+        if (eq) {
+          const unsigned slot = base_slot + __popc(be & ((1u << lane) - 1u));
+          if (slot < (unsigned)SEL_CAND_MAX) pub.cand[slot] = key;
+        }
+      } else {
+        n_eq += __popc(__ballot_sync(0xffffffffu, eq));
+      }
     }
-    gt = __reduce_add_sync(0xffffffffu, gt);
-    eq = __reduce_add_sync(0xffffffffu, eq);
-    if (lane == 0) { atomicAdd(&cta_cnt[0], gt); atomicAdd(&cta_cnt[1], eq); }
+    if (lane == 0) {
+      if (n_above) atomicAdd(&pub.above, n_above);
+      if (n_eq) atomicAdd(&pub.eq, n_eq);
+    }
   }
-  cl.sync();
+  dd_cluster_sync();
+  // ---- F. every block derives the threshold and its own output offsets
+  if (tid < C) {
+    const dd_sel_pub* pr = cl.map_shared_rank(&pub, tid);
+    peer_above[tid] = pr->above;
+    peer_eq[tid] = pr->eq;
+    peer_cand[tid] = min(pr->cand_n, (unsigned)SEL_CAND_MAX);
+  }
+  __syncthreads();
+  uint32_t thr = 0xFFFFFFFFu;
   unsigned base_gt = 0, base_eq = 0;
-  for (int r = 0; r < rank; ++r) {
-    base_gt += *cl.map_shared_rank(&cta_cnt[0], r);
-    base_eq += *cl.map_shared_rank(&cta_cnt[1], r);
-  }
-  int* out = out_idx + bg * k;
-  for (int c0 = 0; c0 < n_local; c0 += SEL_THREADS) {
-    const int pl = c0 + tid;
-    unsigned gt = 0, eq = 0;
-    if (pl < n_local) {
-      const uint32_t key = keys[(size_t)pl * KS];
-      if (p_lo + pl >= n_free || key > thr) gt = 1;
-      else if (key == thr) eq = 1;
+  for (int r = 0; r < rank; ++r) base_gt += peer_above[r];
+  if (k_free > 0 && shift == 0) {
+    thr = klo + (uint32_t)prefix;                 // k_rem of the keys equal to thr are still to be taken
+    for (int r = 0; r < rank; ++r) base_eq += peer_eq[r];
+  } else if (k_free > 0) {
+    unsigned n_all = 0, n_mine_from = 0;          // candidates of all blocks, in block order
+    for (int r = 0; r < C; ++r) {
+      if (r == rank) n_mine_from = n_all;
+      const uint32_t* cr = cl.map_shared_rank(&pub, r)->cand;
+      const unsigned n_r = peer_cand[r];
+      for (unsigned i = tid; i < n_r; i += SEL_THREADS) all_c[n_all + i] = cr[i];
+      n_all += n_r;
     }
-    unsigned total;
-    const unsigned ex = dd_scan256_excl(gt | (eq << 16), warp_tot, total);
-    const unsigned eq_before = base_eq + (ex >> 16);
-    if (gt || (eq && eq_before < k_rem)) {
-      const unsigned pos = base_gt + (ex & 0xFFFFu) + min(eq_before, k_rem);
-      if (pos < (unsigned)k) out[pos] = p_lo + pl;
+    __syncthreads();
+    for (unsigned i = tid; i < n_all; i += SEL_THREADS) {
+      const uint32_t v = all_c[i];
+      unsigned gtc = 0, gec = 0;
+      for (unsigned j = 0; j < n_all; ++j) {
+        const uint32_t u = all_c[j];
+        gtc += u > v;
+        gec += u >= v;
+      }
+      if (gtc < k_rem && k_rem <= gec) { sh_thr = v; sh_above = gtc; }   // equal candidates write equal values
     }
-    base_gt += total & 0xFFFFu;
-    base_eq += total >> 16;
+    __syncthreads();
+    thr = sh_thr;
+    k_rem -= sh_above;
+    // candidates of lower blocks above / equal to the threshold
+    unsigned c_gt = 0, c_eq = 0;
+    for (unsigned i = tid; i < n_mine_from; i += SEL_THREADS) {
+      c_gt += all_c[i] > thr;
+      c_eq += all_c[i] == thr;
+    }
+    c_gt = __reduce_add_sync(0xffffffffu, c_gt);
+    c_eq = __reduce_add_sync(0xffffffffu, c_eq);
+    if (lane == 0) {
+      if (c_gt) atomicAdd(&sh_base_gt, c_gt);
+      if (c_eq) atomicAdd(&sh_base_eq, c_eq);
+    }
+    __syncthreads();
+    base_gt += sh_base_gt;
+    base_eq += sh_base_eq;
   }
-  if (rank == 0)                                 // precondition k <= n_pages violated: pad with the last valid page
-    for (int j = k_eff + tid; j < k; j += SEL_THREADS) out[j] = np > 0 ? np - 1 : 0;
-  cl.sync();                                     // nobody leaves while its shared memory may still be read
+  dd_cluster_arrive();                           // last remote read done: peers may leave
+  // ---- G. ordered compaction of this block's pages: a warp owns a contiguous segment and walks it 32 pages at a
+  // time; ascending page numbers, equal keys are taken from the lowest page up
+  {
+    const int seg = (((n_local + SEL_WARPS - 1) / SEL_WARPS) + 31) & ~31;
+    const int s0 = min(n_local, warp * seg), s1 = min(n_local, s0 + seg);
+    const unsigned lt = (1u << lane) - 1u;
+    unsigned n_gt = 0, n_eq = 0;
+    for (int base = s0; base < s1; base += 32) {
+      const int pl = base + lane;
+      bool gt = false, eq = false;
+      if (pl < s1) {
+        const uint32_t key = keys[pl];
+        gt = p_lo + pl >= n_free || key > thr;
+        eq = !gt && key == thr;
+      }
+      n_gt += __popc(__ballot_sync(0xffffffffu, gt));
+      n_eq += __popc(__ballot_sync(0xffffffffu, eq));
+    }
+    if (lane == 0) { warp_gt[warp] = n_gt; warp_eq[warp] = n_eq; }
+    __syncthreads();
+    unsigned run_gt = base_gt, run_eq = base_eq;
+    for (int w = 0; w < warp; ++w) { run_gt += warp_gt[w]; run_eq += warp_eq[w]; }
+    int* out = out_idx + bg * k;
+    for (int base = s0; base < s1; base += 32) {
+      const int pl = base + lane;
+      bool gt = false, eq = false;
+      if (pl < s1) {
+        const uint32_t key = keys[pl];
+        gt = p_lo + pl >= n_free || key > thr;
+        eq = !gt && key == thr;
+      }
+      const unsigned bgt = __ballot_sync(0xffffffffu, gt), beq = __ballot_sync(0xffffffffu, eq);
+      const unsigned gt_before = run_gt + __popc(bgt & lt);
+      const unsigned eq_before = run_eq + __popc(beq & lt);
+      if (gt || (eq && eq_before < k_rem)) {
+        const unsigned pos = gt_before + min(eq_before, k_rem);
+        if (pos < (unsigned)k) out[pos] = p_lo + pl;
+      }
+      run_gt += __popc(bgt);
+      run_eq += __popc(beq);
+    }
+    if (rank == 0)                               // precondition k <= n_pages violated: pad with the last valid page
+      for (int j = k_eff + tid; j < k; j += SEL_THREADS) out[j] = np > 0 ? np - 1 : 0;
+  }
+  dd_cluster_wait();                             // nobody leaves while its shared memory may still be read
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -696,8 +875,9 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_loads_only_kernel(const __nv_bfloat16* __restrict__ lm,
                                                                               const int* __restrict__ n_pages, int P,
-                                                                              int Hkv, int ppc, int R,
+                                                                              int Hkv, int ppc, int R, int ring_stages,
                                                                               unsigned int* __restrict__ sink) {
+  extern __shared__ __align__(16) unsigned char sel_smem[];
   const int rank = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gl = lane >> 2, t = lane & 3;
@@ -705,35 +885,49 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_loads_only_kernel(co
   const int np = min(n_pages[b], P);
   const int row_lo = rank * ppc * R, row_max = P * R - 1;
   const int n_local_rows = max(0, min(np * R, row_lo + ppc * R) - row_lo);
+  const int n_tiles = (n_local_rows + 15) >> 4;
   const __nv_bfloat16* lm_bg = lm + bg * (size_t)P * R * DD_D;
+  uint4* my_ring = reinterpret_cast<uint4*>(sel_smem) + (size_t)warp * ring_stages * 256 + lane;
   unsigned int acc = 0;
-  for (int t0 = warp * 32; t0 < n_local_rows; t0 += SEL_WARPS * 32) {
-    uint4 lo[2][4], hi[2][4];
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)min(row_lo + t0 + mt * 16 + gl, row_max) * DD_D);
-      const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)min(row_lo + t0 + mt * 16 + gl + 8, row_max) * DD_D);
+  auto issue = [&](int tile, int slot) {
+    if (tile < n_tiles) {
+      const int pa = min(row_lo + tile * 16 + gl, row_max);
+      const int pb = min(row_lo + tile * 16 + gl + 8, row_max);
+      const uint4* ra = reinterpret_cast<const uint4*>(lm_bg + (size_t)pa * DD_D) + t;
+      const uint4* rb = reinterpret_cast<const uint4*>(lm_bg + (size_t)pb * DD_D) + t;
+      uint4* dst = my_ring + slot * 256;
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
-        lo[mt][kk] = dd_ld_stream(ra + kk * 4 + t);
-        hi[mt][kk] = dd_ld_stream(rb + kk * 4 + t);
+        dd_cp_async16(dst + kk * 32, ra + kk * 4);
+        dd_cp_async16(dst + (4 + kk) * 32, rb + kk * 4);
       }
     }
+    dd_cp_async_commit();
+  };
+  const int ahead = ring_stages - 1;
+  for (int s = 0; s < ahead; ++s) issue(warp + s * SEL_WARPS, s);
+  int slot = 0, slot_issue = ahead;
+  for (int tile = warp; tile < n_tiles; tile += SEL_WARPS) {
+    issue(tile + ahead * SEL_WARPS, slot_issue);
+    dd_cp_async_wait_pending(ahead);
+    const uint4* src = my_ring + slot * 256;
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int kk = 0; kk < 4; ++kk)
-        acc ^= lo[mt][kk].x ^ lo[mt][kk].y ^ lo[mt][kk].z ^ lo[mt][kk].w ^ hi[mt][kk].x ^ hi[mt][kk].y ^ hi[mt][kk].z ^
-               hi[mt][kk].w;
+    for (int i = 0; i < 8; ++i) {
+      const uint4 v = src[i * 32];
+      acc ^= v.x ^ v.y ^ v.z ^ v.w;
+    }
+    slot = slot + 1 == ring_stages ? 0 : slot + 1;
+    slot_issue = slot_issue + 1 == ring_stages ? 0 : slot_issue + 1;
   }
+  dd_cp_async_wait_pending(0);
   if (acc == 0x9E3779B9u) sink[0] = acc;        // keeps the loads alive; practically never true
 }
 
 int dd_launch_select_loads_only(dd_ctx* ctx, const void* landmarks, const int* n_pages, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
   if (ctx->sel_cluster <= 0) return dd_fail(ctx, DD_ERR_STATE, "the load-only probe follows the fused selection kernel");
-  dd_select_loads_only_kernel<<<dim3(ctx->sel_cluster, c.n_kv_heads, c.batch), SEL_THREADS, 0, st>>>(
-      (const __nv_bfloat16*)landmarks, n_pages, c.max_pages, c.n_kv_heads, ctx->sel_ppc, ctx->R,
+  dd_select_loads_only_kernel<<<dim3(ctx->sel_cluster, c.n_kv_heads, c.batch), SEL_THREADS, ctx->sel_smem_bytes, st>>>(
+      (const __nv_bfloat16*)landmarks, n_pages, c.max_pages, c.n_kv_heads, ctx->sel_ppc, ctx->R, ctx->sel_stages,
       ctx->attn_ticket + c.batch * c.n_kv_heads);
   DD_CUDA_TRY(ctx, cudaGetLastError());
   return DD_OK;
@@ -745,6 +939,13 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
   const int G = ctx->G;
   if (ctx->R > 1 && !ctx_len) return dd_fail(ctx, DD_ERR_INVALID_ARG, "finer landmarks need ctx_len for the selection");
   if (ctx->sel_cluster > 0) {
+    // logits in global scratch: the selection stream of the pipelined path has a buffer of its own, because a
+    // selection there may run next to one on the compute stream
+    float* s_glob = nullptr;
+    if (ctx->sel_logits_global) {
+      const size_t per_buf = (size_t)c.batch * c.n_kv_heads * c.max_pages * ctx->R * G;
+      s_glob = ctx->score_s + ((c.select_stream && st == (cudaStream_t)c.select_stream) ? per_buf : 0);
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(ctx->sel_cluster, c.n_kv_heads, c.batch);
     cfg.blockDim = dim3(SEL_THREADS);
@@ -761,7 +962,7 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
                                         q_tokens_in_tensor * c.n_q_heads * DD_D, q_token * c.n_q_heads * DD_D,
                                         (const __nv_bfloat16*)landmarks, n_pages, out_idx, out_scores, c.max_pages, G,
                                         c.n_kv_heads, c.k_pages, c.forced_recent_pages, ctx->sel_ppc, ctx->err_word,
-                                        ctx->R, ctx_len));
+                                        ctx->R, ctx_len, ctx->sel_stages, s_glob));
     return DD_OK;
   }
   dim3 sgrid(ctx->score_tiles, c.n_kv_heads, c.batch);
@@ -782,9 +983,32 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
 // (two blocks per SM), every block has at least 32 pages, and a block's share of the logits fits in shared
 // memory. Up to 8 blocks, 16 for very long requests. 0 = not possible, use the two-kernel path.
 // The search walks a fixed candidate list exactly once, so it always terminates; `fits` answers whether clusters of that shape can be resident on the device.
+// Shared memory of one block: the logits of its rows (unless they live in global scratch), then the larger of the
+// scoring ring (one 4 KiB tile per warp and stage) and the keys + two histograms that take its place afterwards.
+static size_t dd_select_smem(int ppc, int rows_per_page, int group, int stages, bool logits_in_smem) {
+  const size_t ring = (size_t)SEL_WARPS * stages * 4096, later = (size_t)ppc * 4 + 2 * RADIX_BINS * 4;
+  return (logits_in_smem ? (size_t)ppc * rows_per_page * group * 4 : 0) + (ring > later ? ring : later);
+}
+
+// Block shape of the fused selection for one cluster size: every block is sized so that two fit on an SM (the device
+// holds about half as many clusters otherwise). The logits stay in shared memory when a ring of two tiles per warp
+// still fits next to them; else they go to global scratch.
+static void dd_select_shape(int max_pages, int C, int rows_per_page, int group, int* ppc_out, int* stages_out,
+                            int* logits_global_out, size_t* smem_out) {
+  const size_t budget = (size_t)112 * 1024;
+  int ppc = (max_pages + C - 1) / C;
+  ppc = (ppc + 31) & ~31;                                  // whole pairs of MMA tiles
+  const bool in_smem = dd_select_smem(ppc, rows_per_page, group, 2, true) <= budget;
+  const int stages = 2;                                    // measured: deeper rings buy nothing, larger blocks launch slower
+  *ppc_out = ppc;
+  *stages_out = stages;
+  *logits_global_out = in_smem ? 0 : 1;
+  *smem_out = dd_select_smem(ppc, rows_per_page, group, stages, in_smem);
+}
+
 extern "C" int dd_test_pick_cluster(int max_pages, int problems, int sm_count, int rows_per_page, int group, int allow16,
                                     int (*fits)(int blocks, size_t shared_bytes, void* user), void* user,
-                                    int* pages_per_block, size_t* shared_bytes) {
+                                    int* pages_per_block, size_t* shared_bytes, int* ring_stages, int* logits_global) {
   if (max_pages < 1 || problems < 1 || sm_count < 1 || rows_per_page < 1 || group < 1 || !fits) return 0;
   const int c_max = (max_pages >= 32768 && allow16) ? 16 : 8;
   int start = 1;
@@ -793,22 +1017,27 @@ extern "C" int dd_test_pick_cluster(int max_pages, int problems, int sm_count, i
   int cand[16], n_cand = 0;
   for (int C = start; C <= c_max; C *= 2) cand[n_cand++] = C;
   for (int C = start / 2; C >= 1; C /= 2) cand[n_cand++] = C;
-  for (int i = 0; i < n_cand; ++i) {
-    const int C = cand[i];
-    int ppc = (max_pages + C - 1) / C;
-    ppc = (ppc + 31) & ~31;                                // whole pairs of MMA tiles
-    const size_t smem = (size_t)ppc * rows_per_page * group * 4 + 2 * RADIX_BINS * 4;
-    if (smem > (size_t)SEL_MAX_SMEM) continue;             // too long for this cluster size
-    if (!fits(C, smem, user)) continue;
-    if (pages_per_block) *pages_per_block = ppc;
-    if (shared_bytes) *shared_bytes = smem;
-    return C;
+  // first choice: a size of which the device holds all clusters at once; else any size that can run at all
+  for (int need_all = 1; need_all >= 0; --need_all) {
+    for (int i = 0; i < n_cand; ++i) {
+      const int C = cand[i];
+      int ppc, stages, lg;
+      size_t smem;
+      dd_select_shape(max_pages, C, rows_per_page, group, &ppc, &stages, &lg, &smem);
+      if (smem > (size_t)SEL_MAX_SMEM) continue;           // too long for this cluster size
+      if (fits(C, smem, user) < (need_all ? problems : 1)) continue;
+      if (pages_per_block) *pages_per_block = ppc;
+      if (shared_bytes) *shared_bytes = smem;
+      if (ring_stages) *ring_stages = stages;
+      if (logits_global) *logits_global = lg;
+      return C;
+    }
   }
   return 0;
 }
 
-static int dd_select_cluster_fits(int C, size_t smem, void* user) {
-  const dd_ctx* ctx = (const dd_ctx*)user;
+// How many clusters of C blocks with `smem` bytes of dynamic shared memory can be resident at once (0 on error).
+static int dd_select_resident_clusters(const dd_ctx* ctx, int C, size_t smem) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(C, ctx->cfg.n_kv_heads, ctx->cfg.batch);
   cfg.blockDim = dim3(SEL_THREADS);
@@ -825,7 +1054,11 @@ static int dd_select_cluster_fits(int C, size_t smem, void* user) {
     cudaGetLastError();
     return 0;
   }
-  return n_clusters >= 1;
+  return n_clusters;
+}
+
+static int dd_select_cluster_fits(int C, size_t smem, void* user) {
+  return dd_select_resident_clusters((const dd_ctx*)user, C, smem);
 }
 
 static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
@@ -838,7 +1071,7 @@ static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
   if (!big_ok) cudaGetLastError();
   size_t smem = 0;
   const int C = dd_test_pick_cluster(c.max_pages, c.batch * c.n_kv_heads, ctx->sm_count, ctx->R, ctx->G, big_ok ? 1 : 0,
-                                     dd_select_cluster_fits, ctx, ppc_out, &smem);
+                                     dd_select_cluster_fits, ctx, ppc_out, &smem, &ctx->sel_stages, &ctx->sel_logits_global);
   *smem_out = (int)smem;
   return C;
 }
@@ -846,6 +1079,8 @@ static int dd_select_pick_cluster(dd_ctx* ctx, int* ppc_out, int* smem_out) {
 int dd_select_setup(dd_ctx* ctx) {
   DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(TOPK_SMEM_KEYS * sizeof(uint32_t))));
+  DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_select_loads_only_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        SEL_MAX_SMEM));
   ctx->sel_cluster = 0;
   if (ctx->cfg.select_mode != DD_SELECT_TWO_KERNELS)
     ctx->sel_cluster = dd_select_pick_cluster(ctx, &ctx->sel_ppc, &ctx->sel_smem_bytes);

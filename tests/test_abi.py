@@ -42,42 +42,48 @@ def test_binding_lists_the_same_entry_points_and_error_strings():
 
 
 def test_cluster_search_of_the_fused_selection_always_terminates():
-    """The search over cluster sizes with the device queries replaced by a callback: whatever the callback
-    answers, the search ends, and it returns 0 (two-kernel path) when nothing fits."""
+    """The search over cluster sizes with the device queries replaced by a callback (how many clusters of a
+    shape are resident at once): whatever the callback answers, the search ends; it prefers a size whose
+    clusters are all resident, and returns 0 (two-kernel path) when nothing can run."""
     from paper_2607_26475_b200 import build
     build.build()
     from paper_2607_26475_b200 import binding
-    ppc, smem = ctypes.c_int(), ctypes.c_size_t()
+    ppc, smem, stages, lg = ctypes.c_int(), ctypes.c_size_t(), ctypes.c_int(), ctypes.c_int()
 
     def pick(max_pages, problems, rows, allow16, answer):
         calls = []
 
         def fits(c, sm, _):
             calls.append((c, sm))
-            assert len(calls) < 16, "the search does not terminate"
-            return 1 if answer(c, sm) else 0
+            assert len(calls) < 32, "the search does not terminate"
+            return int(answer(c, sm))
         cb = binding.PICK_FITS(fits)
-        got = binding.lib.dd_test_pick_cluster(max_pages, problems, 148, rows, 4, allow16, cb, None,
-                                                ctypes.byref(ppc), ctypes.byref(smem))
+        got = binding.lib.dd_test_pick_cluster(max_pages, problems, 148, rows, 4, allow16, cb, None, ctypes.byref(ppc),
+                                                ctypes.byref(smem), ctypes.byref(stages), ctypes.byref(lg))
         return got, calls
 
-    # config 2: 64 problems of 2048 pages -> 4 blocks each, 512 pages per block
-    got, calls = pick(2048, 64, 1, 1, lambda c, s: True)
-    assert got == 4 and ppc.value == 512 and smem.value == 512 * 4 * 4 + 2 * 2048 * 4
-    # one request of 64K pages: 16-block clusters when allowed, 8 otherwise
-    assert pick(65536, 8, 1, 1, lambda c, s: True)[0] == 16
-    assert pick(65536, 8, 1, 0, lambda c, s: True)[0] == 8
-    # 16 refused by the device: 8 is tried next, once
-    got, calls = pick(65536, 8, 1, 1, lambda c, s: c != 16)
-    assert got == 8 and [c for c, _ in calls] == [16, 8]
-    # the case that used to loop: 128K pages with four landmarks per page; 8 blocks exceed shared memory and
-    # the device refuses 16-block clusters
-    got, calls = pick(131072, 8, 4, 1, lambda c, s: False)
-    assert got == 0 and len(calls) <= 5
-    got, calls = pick(131072, 8, 1, 1, lambda c, s: False)
-    assert got == 0 and len(calls) <= 5
-    # nothing ever fits
-    assert pick(2048, 64, 1, 1, lambda c, s: False)[0] == 0
-    # a larger cluster is used when the preferred one does not fit
-    got, calls = pick(2048, 64, 1, 1, lambda c, s: c >= 8)
+    # what a B200 answers for blocks of at most 112 KiB (two per SM)
+    b200 = {1: 296, 2: 148, 4: 71, 8: 33, 16: 14}
+    # batch 8 x 8 KV heads, 2048 pages: 4 blocks each, 512 pages per block, logits in shared memory, 3-tile ring
+    got, calls = pick(2048, 64, 1, 1, lambda c, s: b200[c])
+    assert got == 4 and ppc.value == 512 and stages.value == 2 and lg.value == 0
+    assert smem.value == 512 * 4 * 4 + 8 * 2 * 4096 and smem.value <= 112 * 1024
+    # one request of 64K pages: 16-block clusters, logits in global scratch, every block small enough for two per SM
+    got, _ = pick(65536, 8, 1, 1, lambda c, s: b200[c])
+    assert got == 16 and ppc.value == 4096 and lg.value == 1 and smem.value <= 112 * 1024 and stages.value == 2
+    assert pick(65536, 8, 1, 0, lambda c, s: b200[c])[0] == 8
+    # 16 refused by the device: 8 is tried next, once per round
+    got, calls = pick(65536, 8, 1, 1, lambda c, s: 0 if c == 16 else b200[c])
+    assert got == 8 and [c for c, _ in calls][:2] == [16, 8]
+    # not all clusters resident for any size: the preferred size is taken in the second round
+    got, calls = pick(2048, 64, 1, 1, lambda c, s: 1)
+    assert got == 4 and len(calls) <= 10
+    # the case that used to loop: 128K pages with four landmarks per page, and a device that refuses everything
+    got, calls = pick(131072, 8, 4, 1, lambda c, s: 0)
+    assert got == 0 and len(calls) <= 10
+    got, calls = pick(131072, 8, 1, 1, lambda c, s: 0)
+    assert got == 0 and len(calls) <= 10
+    assert pick(2048, 64, 1, 1, lambda c, s: 0)[0] == 0
+    # a larger cluster is used when the preferred one cannot hold all its clusters
+    got, calls = pick(2048, 64, 1, 1, lambda c, s: 64 if c >= 8 else 10)
     assert got == 8 and [c for c, _ in calls] == [4, 8]
