@@ -29,6 +29,9 @@ DD_GATHER_BULK = 1
 DD_GATHER_STAGED = 2
 DD_GATHER_STATS_FIELDS = 7
 DD_TRACE_FIELDS = 8
+DD_ATTN_AUTO = 0
+DD_ATTN_SPLIT = 1
+DD_ATTN_STREAM = 2
 DD_SELECT_AUTO = 0
 DD_SELECT_TWO_KERNELS = 1
 
@@ -54,7 +57,7 @@ class DDConfig(C.Structure):
         ("compute_stream", C.c_void_p), ("copy_stream", C.c_void_p),
         ("ring_mem", C.c_void_p), ("ring_bytes", C.c_size_t),
         ("landmark_chunk_tokens", C.c_int), ("miss_correction", C.c_int), ("urgent_stream", C.c_void_p),
-        ("select_stream", C.c_void_p), ("stage_min_run_pages", C.c_int), ("stage_block_pages", C.c_int),
+        ("select_stream", C.c_void_p), ("stage_min_run_pages", C.c_int), ("stage_block_pages", C.c_int), ("attn_mode", C.c_int),
     ]
 
 
@@ -174,7 +177,7 @@ class Context:
                  page_tokens=16, forced_recent_pages=0, n_q_tokens=2, ring_depth=2, gather_mode=DD_GATHER_LOADS,
                  gather_ctas=0, select_mode=DD_SELECT_AUTO, attn_splits=0, compute_stream=None, copy_stream=None, ring=None,
                  miss_correction=False, urgent_stream=None, landmark_chunk_tokens=0, select_stream=None,
-                 stage_min_run_pages=0, stage_block_pages=0):
+                 stage_min_run_pages=0, stage_block_pages=0, attn_mode=DD_ATTN_AUTO):
         if not torch.cuda.is_available():
             raise RuntimeError("the sparse decode path needs a CUDA device; there is no CPU fallback")
         self.compute_stream = compute_stream if compute_stream is not None else torch.cuda.current_stream()
@@ -190,7 +193,7 @@ class Context:
                             landmark_chunk_tokens, 1 if miss_correction else 0,
                             self.urgent_stream.cuda_stream if self.urgent_stream is not None else None,
                             select_stream.cuda_stream if select_stream is not None else None,
-                            stage_min_run_pages, stage_block_pages)
+                            stage_min_run_pages, stage_block_pages, attn_mode)
         self.select_stream = select_stream
         self._h = C.c_void_p()
         self._keep = []

@@ -70,6 +70,7 @@ static const char* dd_check_config(const dd_config* c) {
     const int ct = c->landmark_chunk_tokens;
     if (ct != 0 && ct != 16 && ct != 8 && ct != 4 && ct != 2 && ct != 1) return "landmark_chunk_tokens must be 0, 16, 8, 4, 2 or 1";
   }
+  if (c->attn_mode != DD_ATTN_AUTO && c->attn_mode != DD_ATTN_SPLIT && c->attn_mode != DD_ATTN_STREAM) return "unknown attn_mode";
   if (c->attn_splits > 512) return "attn_splits must be <= 512";
   if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";
   if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
@@ -116,7 +117,7 @@ struct dd_sizes {
 
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
+static dd_sizes dd_compute_sizes(const dd_config* c, int S, int sm_count) {
   dd_sizes z;
   const size_t B = c->batch, Hkv = c->n_kv_heads, Hq = c->n_q_heads, P = c->max_pages;
   const size_t G = Hq / Hkv, tiles = (P + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
@@ -124,8 +125,14 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S) {
   z.score_s = up256(2 * B * Hkv * P * Rr * G * 4);
   z.score_part = up256(B * Hq * tiles * 8);
   z.topk_keys = up256(B * Hkv * P * 4);
-  z.part_o = up256(B * Hkv * (size_t)S * 8 * DD_D * 4);
-  z.part_ml = up256(B * Hkv * (size_t)S * 8 * 8);
+  {
+    // partials of the split-KV kernel (S per unit) or of the streaming kernel (max_parts per unit), whichever is larger
+    int nb = 0, ppb = 0, parts = 0;
+    dd_attn_stream_geometry(c, sm_count, &nb, &ppb, &parts);
+    const size_t n_part = (size_t)(S > parts ? S : parts);
+    z.part_o = up256(B * Hkv * n_part * 8 * DD_D * 4);
+    z.part_ml = up256(B * Hkv * n_part * 8 * 8);
+  }
   z.ticket = up256(B * Hkv * 4 + 4);               // arrival counters + one word the load-only probes may write
   z.idx_tab = up256((size_t)2 * c->n_layers * B * Hkv * c->k_pages * 4);
   z.err = 256;
@@ -154,7 +161,7 @@ extern "C" size_t dd_slot_bytes(const dd_config* c) {
 extern "C" size_t dd_ring_bytes(const dd_config* c) { return dd_slot_bytes(c) * (c ? (size_t)c->ring_depth : 0); }
 extern "C" size_t dd_scratch_bytes(const dd_config* c) {
   if (dd_check_config(c)) return 0;
-  return dd_compute_sizes(c, dd_resolve_splits(c, dd_sm_count(), nullptr)).total();
+  return dd_compute_sizes(c, dd_resolve_splits(c, dd_sm_count(), nullptr), dd_sm_count()).total();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -226,7 +233,7 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   ctx->score_tiles = (cfg->max_pages + DD_SCORE_TILE - 1) / DD_SCORE_TILE;
   ctx->attn_splits = dd_resolve_splits(cfg, ctx->sm_count, &ctx->attn_cluster);
   ctx->slot_bytes = dd_slot_bytes(cfg);
-  const dd_sizes z = dd_compute_sizes(cfg, ctx->attn_splits);
+  const dd_sizes z = dd_compute_sizes(cfg, ctx->attn_splits, ctx->sm_count);
 
 #define DD_CREATE_TRY(expr)                                                                        \
   do {                                                                                             \
@@ -324,6 +331,8 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   }
   int rc = dd_select_setup(ctx);
   if (rc == DD_OK) rc = dd_gather_setup(ctx);
+  ctx->attn_stream = cfg->attn_mode == DD_ATTN_STREAM;   // measured slower than the split-KV kernel: opt-in only
+  if (rc == DD_OK && ctx->attn_stream) rc = dd_attn_stream_setup(ctx);
   if (rc != DD_OK) {
     memcpy(g_errmsg, ctx->errmsg, 512);
     dd_free_all(ctx);

@@ -1,0 +1,540 @@
+// GQA decode attention over the gathered set of a ring slot, streaming form.
+//
+// The slot of a layer is one long list of pages (B * Hkv units of k pages each). It is cut into equal runs of
+// consecutive pages, one per thread block, two blocks per SM, regardless of where the unit boundaries fall: every
+// SM streams the same number of bytes. Inside a block one producer thread keeps a ring of pages in flight with
+// tiled bulk-tensor copies (TMA, 128-byte swizzle, completion on mbarriers); four consumer warps take pages from
+// the ring, read their MMA fragments from shared memory without bank conflicts, and run the same transposed
+// bf16 MMA formulation as dd_attn_kernel (the up-to-8 query rows of a KV head are the N = 8 columns). When a
+// block's run crosses into the next unit the consumers merge and publish what they have for the unit they leave;
+// units that were cut across blocks are merged by the last block to arrive (arrival counter, no waiting).
+// Every wait on an mbarrier is bounded; a wait that gives up sets the device error word and the block finishes
+// its control flow without waiting again.
+#include <cuda.h>
+
+#include "dd_common.cuh"
+
+#pragma nv_diag_suppress 128   // the load-only instantiation leaves the merge code unreachable
+
+constexpr int AS_CONSUMERS = 4;                       // consumer warps
+constexpr int AS_THREADS = (AS_CONSUMERS + 1) * 32;   // plus the producer warp
+constexpr int AS_STAGES = 10;                         // pages in flight per block (8 KiB each)
+constexpr int AS_STAGE_BYTES = DD_PAGE_BYTES;         // K channels 0-63, K 64-127, V 0-63, V 64-127: 2 KiB boxes
+constexpr int AS_ROWS = 8;                            // query rows per KV head the MMA shape carries
+constexpr int AS_OPAD = 9;
+constexpr int AS_MAX_PARTS = 64;                      // blocks a unit may be cut across
+constexpr int AS_SMEM_BYTES = AS_STAGES * AS_STAGE_BYTES + 1024;   // + slack to align the ring to 1 KiB
+
+__device__ __forceinline__ uint32_t as_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long as_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait for a phase of an mbarrier. Returns at once when another thread of the block already gave up.
+__device__ __forceinline__ bool as_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned long long limit_ns) {
+  unsigned long long t0 = 0;
+  for (unsigned it = 0;; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (*abort_flag) return false;
+    if ((it & 31u) == 31u) {
+      const unsigned long long now = as_timer();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+__device__ __forceinline__ void as_tma_box(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tmap), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ uint32_t as_movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+
+__device__ __forceinline__ uint32_t as_pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint32_t as_word(const uint4& v, int w) {
+  return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+}
+
+__device__ __forceinline__ uint4 as_lds(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+// Fragments of the page in ring stage `st` (shared-memory address). A box is [16 tokens][64 channels] with
+// 128-byte rows whose 16-byte chunks are XOR-swizzled with the row number (mod 8).
+//   K: rows gl and gl + 8; k-step kk takes chunk 2t + (kk & 1) of the half kk >> 1 (any fixed assignment of the 128
+//      channels to k-slots is fine as long as the query fragment uses the same one); conflict-free because the two
+//      rows of a quarter-warp are an even and an odd row, whose XOR keeps the chunk sets apart.
+//   V: tokens 2t, 2t+1, 2t+8, 2t+9; chunk gl of both halves.
+__device__ __forceinline__ void as_load_frags(uint32_t st, int gl, int t, uint4 (&klo)[4], uint4 (&khi)[4], uint4 (&v)[4][2]) {
+#pragma unroll
+  for (int kk = 0; kk < 4; ++kk) {
+    const uint32_t box = st + (kk >> 1) * 2048;
+    const uint32_t ch = (uint32_t)((2 * t + (kk & 1)) ^ gl) << 4;
+    klo[kk] = as_lds(box + gl * 128 + ch);
+    khi[kk] = as_lds(box + (gl + 8) * 128 + ch);
+  }
+#pragma unroll
+  for (int tk = 0; tk < 4; ++tk) {
+    const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
+    const uint32_t ch = (uint32_t)(gl ^ (tok & 7)) << 4;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) v[tk][c] = as_lds(st + 4096 + c * 2048 + tok * 128 + ch);
+  }
+}
+
+// Grid: n_blocks blocks of AS_THREADS threads; block x owns the pages [x * ppb, min(total, (x + 1) * ppb)) of the
+// flat list (unit u = page / k, position j = page % k). part_o / part_ml hold max_parts partials per unit.
+template <bool PROBE>
+__global__ void __launch_bounds__(AS_THREADS, 2) dd_attn_stream_kernel(
+    const __grid_constant__ CUtensorMap tmap, const __nv_bfloat16* __restrict__ q, const int* __restrict__ idx,
+    const int* __restrict__ ctx_len, __nv_bfloat16* __restrict__ out, float* __restrict__ out_lse,
+    float* __restrict__ part_o, float2* __restrict__ part_ml, unsigned int* __restrict__ ticket, int Hkv, int G, int Tq,
+    int k, int total_pages, int ppb, int max_parts, const __nv_bfloat16* __restrict__ k_new,
+    const __nv_bfloat16* __restrict__ v_new, int* err_word, unsigned long long wait_ns, unsigned int* __restrict__ sink) {
+  extern __shared__ unsigned char as_dyn[];
+  __shared__ __align__(8) unsigned long long full_bar[AS_STAGES];
+  __shared__ __align__(8) unsigned long long empty_bar[AS_STAGES];
+  __shared__ float sm_o[AS_CONSUMERS][DD_D][AS_OPAD];   // per-warp O^T, [channel][row]
+  __shared__ float2 sm_ml[AS_CONSUMERS][AS_ROWS];
+  __shared__ float sm_scale[AS_CONSUMERS][AS_ROWS];
+  __shared__ float2 blk_ml[AS_ROWS];
+  __shared__ int sm_last;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gl = lane >> 2, t = lane & 3;
+  const uint32_t ring = (as_smem(as_dyn) + 1023u) & ~1023u;          // swizzled boxes want 1 KiB alignment
+  const int f0 = blockIdx.x * ppb;
+  const int f1 = min(total_pages, f0 + ppb);
+  const int n_mine = f1 - f0;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < AS_STAGES; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(as_smem(&full_bar[s])));
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(as_smem(&empty_bar[s])));
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_p = &abort_flag;
+
+  if (warp == AS_CONSUMERS) {
+    // ---- producer: one thread keeps the ring full
+    if (lane == 0) {
+      int issued = 0;
+      for (int i = 0; i < n_mine; ++i) {
+        const int s = i % AS_STAGES, round = i / AS_STAGES;
+        if (round > 0 && !as_wait(as_smem(&empty_bar[s]), (uint32_t)((round - 1) & 1), abort_p, wait_ns)) break;
+        const int f = f0 + i;
+        const int u = f / k, j = f - u * k;
+        const int row_k = (u * 2 * k + j) * DD_T, row_v = row_k + k * DD_T;
+        const uint32_t bar = as_smem(&full_bar[s]);
+        const uint32_t dst = ring + (uint32_t)s * AS_STAGE_BYTES;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)AS_STAGE_BYTES) : "memory");
+        as_tma_box(dst, &tmap, 0, row_k, bar);
+        as_tma_box(dst + 2048, &tmap, 64, row_k, bar);
+        as_tma_box(dst + 4096, &tmap, 0, row_v, bar);
+        as_tma_box(dst + 6144, &tmap, 64, row_v, bar);
+        issued = i + 1;
+      }
+      // every copy this thread issued must have landed before the block may retire: wait (bounded, whatever the
+      // abort flag says) for the last use of every stage
+      for (int i = max(0, issued - AS_STAGES); i < issued; ++i) {
+        const uint32_t bar = as_smem(&full_bar[i % AS_STAGES]);
+        const unsigned long long t0 = as_timer();
+        for (unsigned it = 0;; ++it) {
+          uint32_t done;
+          asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                       : "=r"(done) : "r"(bar), "r"((uint32_t)((i / AS_STAGES) & 1)) : "memory");
+          if (done) break;
+          if ((it & 31u) == 31u && as_timer() - t0 > wait_ns) { *abort_p = 1; break; }
+        }
+      }
+      if (*abort_p) dd_report(err_word, DD_ERR_WAIT_EXPIRED, 2);
+    }
+    return;
+  }
+
+  // ---- consumers
+  const int Hq = Hkv * G;
+  const int n_rows = Tq * G;
+  const float scale_log2 = rsqrtf((float)DD_D) * 1.4426950408889634f;
+  const int d = threadIdx.x;                       // the channel a consumer thread owns in the merges (0..127)
+  unsigned int probe_acc = 0;
+  int i_base = 0;                                  // index inside the block's run of the segment's first page
+  for (int f = f0; f < f1;) {
+    const int u = f / k, j0 = f - u * k;
+    const int seg_n = min(f1 - f, k - j0);
+    const int b = u / Hkv, g = u - b * Hkv;
+    const size_t bg = (size_t)u;
+    // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G), channels in the K fragment's order
+    uint4 qf[4];
+    if (!PROBE && gl < n_rows) {
+      const int tq = gl / G, hh = gl - tq * G;
+      const uint4* qrow = reinterpret_cast<const uint4*>(q + (((size_t)b * Tq + tq) * Hq + g * G + hh) * DD_D);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = __ldg(qrow + (kk >> 1) * 8 + 2 * t + (kk & 1));
+    } else {
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) qf[kk] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const int* idx_bg = idx + bg * k;
+    const int n_ctx = PROBE ? 0 : ctx_len[b];
+
+    float o[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY};   // columns n = 2t, 2t+1, log2 domain
+    float l_run[2] = {0.f, 0.f};               // partial over this lane's tokens
+    uint4 klo[4], khi[4], v[4][2];
+
+    auto qk = [&](float (&acc)[4]) {
+      float acc2[4] = {0.f, 0.f, 0.f, 0.f};    // two chains: the MMAs of a chain depend on each other
+      acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        dd_mma_bf16(acc, klo[kk].x, khi[kk].x, klo[kk].y, khi[kk].y, qf[kk].x, qf[kk].y);
+        dd_mma_bf16(acc2, klo[kk].z, khi[kk].z, klo[kk].w, khi[kk].w, qf[kk].z, qf[kk].w);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] = (acc[i] + acc2[i]) * scale_log2;
+    };
+    auto softmax_pv = [&](float (&acc)[4]) {
+      float alpha[2], pr[4];
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float pm = fmaxf(acc[c], acc[2 + c]);
+        pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 4));
+        pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 8));
+        pm = fmaxf(pm, __shfl_xor_sync(0xffffffffu, pm, 16));
+        const float mn = fmaxf(m_run[c], pm);
+        if (mn == -INFINITY) {
+          alpha[c] = 1.f; pr[c] = 0.f; pr[2 + c] = 0.f;
+        } else {
+          alpha[c] = exp2f(m_run[c] - mn);
+          pr[c] = exp2f(acc[c] - mn);
+          pr[2 + c] = exp2f(acc[2 + c] - mn);
+        }
+        l_run[c] = l_run[c] * alpha[c] + pr[c] + pr[2 + c];
+        m_run[c] = mn;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        o[i][0] *= alpha[0]; o[i][1] *= alpha[1]; o[i][2] *= alpha[0]; o[i][3] *= alpha[1];
+      }
+      const uint32_t pb0 = as_movmatrix_trans(as_pack_bf16(pr[0], pr[1]));
+      const uint32_t pb1 = as_movmatrix_trans(as_pack_bf16(pr[2], pr[3]));
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {            // MMA tile i: rows gl -> channel 8gl+i, gl+8 -> channel 64+8gl+i
+        const int w = i >> 1;
+        const uint32_t sel = (i & 1) ? 0x7632u : 0x5410u;
+        const uint32_t a0 = __byte_perm(as_word(v[0][0], w), as_word(v[1][0], w), sel);
+        const uint32_t a1 = __byte_perm(as_word(v[0][1], w), as_word(v[1][1], w), sel);
+        const uint32_t a2 = __byte_perm(as_word(v[2][0], w), as_word(v[3][0], w), sel);
+        const uint32_t a3 = __byte_perm(as_word(v[2][1], w), as_word(v[3][1], w), sel);
+        dd_mma_bf16(o[i], a0, a1, a2, a3, pb0, pb1);
+      }
+    };
+
+    if (!PROBE && k_new != nullptr && j0 == 0 && warp == 0) {
+      // the step's own new KV entries (dual-token causal tail): one extra "page" whose tokens 0..Tq-1 are the new
+      // entries; query token t sees the entries j <= t. Taken by the first warp of the block that holds page 0.
+      const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        klo[kk] = gl < Tq ? __ldg(reinterpret_cast<const uint4*>(k_new + (((size_t)b * Tq + gl) * Hkv + g) * DD_D) +
+                                  (kk >> 1) * 8 + 2 * t + (kk & 1))
+                          : zero;
+        khi[kk] = zero;
+      }
+#pragma unroll
+      for (int tk = 0; tk < 4; ++tk) {
+        const int tok = 2 * t + (tk & 1) + (tk >> 1) * 8;
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+          v[tk][c] = tok < Tq ? __ldg(reinterpret_cast<const uint4*>(v_new + (((size_t)b * Tq + tok) * Hkv + g) * DD_D +
+                                                                    c * 64 + gl * 8))
+                              : zero;
+      }
+      float acc[4];
+      qk(acc);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const int n = 2 * t + c;
+        const bool visible = gl < Tq && n < n_rows && gl <= n / G;
+        if (!visible) acc[c] = -INFINITY;
+        acc[2 + c] = -INFINITY;
+      }
+      softmax_pv(acc);
+    }
+
+    // pages of this segment: page ii of the block's run goes to consumer warp ii % AS_CONSUMERS
+    int ii = i_base + ((warp - i_base) % AS_CONSUMERS + AS_CONSUMERS) % AS_CONSUMERS;
+    int page = (!PROBE && ii < i_base + seg_n) ? idx_bg[j0 + ii - i_base] : 0;
+    for (; ii < i_base + seg_n; ii += AS_CONSUMERS) {
+      const int s = ii % AS_STAGES;
+      const int nxt = ii + AS_CONSUMERS;
+      const int page_next = (!PROBE && nxt < i_base + seg_n) ? idx_bg[j0 + nxt - i_base] : 0;
+      // Copies complete in any order, and a warp that is done with its earlier pages may get here while the stage's
+      // previous use (another warp's page) is still in flight. A parity wait on the "full" barrier cannot tell "this
+      // round is complete" from "the round before the previous one is", so first make sure the previous round was
+      // released (that wait is unambiguous: the previous round was issued before any page this warp has seen).
+      const int round = ii / AS_STAGES;
+      if (round > 0) as_wait(as_smem(&empty_bar[s]), (uint32_t)((round - 1) & 1), abort_p, wait_ns);
+      as_wait(as_smem(&full_bar[s]), (uint32_t)(round & 1), abort_p, wait_ns);
+      as_load_frags(ring + (uint32_t)s * AS_STAGE_BYTES, gl, t, klo, khi, v);
+      if (PROBE) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          probe_acc ^= klo[i].x ^ klo[i].w ^ khi[i].y ^ khi[i].z ^ v[i][0].x ^ v[i][0].w ^ v[i][1].y ^ v[i][1].z;
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(as_smem(&empty_bar[s])) : "memory");
+      if (!PROBE) {
+        float acc[4];
+        qk(acc);
+        if (page * DD_T + DD_T > n_ctx) {          // only the last page of a request can be partial
+          if (page * DD_T + gl >= n_ctx) acc[0] = acc[1] = -INFINITY;
+          if (page * DD_T + gl + 8 >= n_ctx) acc[2] = acc[3] = -INFINITY;
+        }
+        softmax_pv(acc);
+      }
+      page = page_next;
+    }
+    f += seg_n;
+    i_base += seg_n;
+    if (PROBE) continue;
+
+    // ---- the segment is done: merge the consumer warps, then publish or finish the unit
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 4);
+      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 8);
+      l_run[c] += __shfl_xor_sync(0xffffffffu, l_run[c], 16);
+    }
+    if (gl == 0) {
+      sm_ml[warp][2 * t] = make_float2(m_run[0], l_run[0]);
+      sm_ml[warp][2 * t + 1] = make_float2(m_run[1], l_run[1]);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      sm_o[warp][8 * gl + i][2 * t] = o[i][0];
+      sm_o[warp][8 * gl + i][2 * t + 1] = o[i][1];
+      sm_o[warp][64 + 8 * gl + i][2 * t] = o[i][2];
+      sm_o[warp][64 + 8 * gl + i][2 * t + 1] = o[i][3];
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (threadIdx.x < AS_ROWS) {
+      const int n = threadIdx.x;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < AS_CONSUMERS; ++w) M = fmaxf(M, sm_ml[w][n].x);
+      float L = 0.f;
+#pragma unroll
+      for (int w = 0; w < AS_CONSUMERS; ++w) {
+        const float sc = (M == -INFINITY) ? 0.f : exp2f(sm_ml[w][n].x - M);
+        sm_scale[w][n] = sc;
+        L += sm_ml[w][n].y * sc;
+      }
+      blk_ml[n] = make_float2(M, L);
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    float ob[AS_ROWS];
+#pragma unroll
+    for (int n = 0; n < AS_ROWS; ++n) {
+      float a = 0.f;
+#pragma unroll
+      for (int w = 0; w < AS_CONSUMERS; ++w) a += sm_o[w][d][n] * sm_scale[w][n];
+      ob[n] = a;
+    }
+    // which blocks hold pages of this unit
+    const int b_first = (u * k) / ppb, b_last = ((u + 1) * k - 1) / ppb;
+    const int n_parts = b_last - b_first + 1;
+    if (n_parts == 1) {
+#pragma unroll
+      for (int n = 0; n < AS_ROWS; ++n) {
+        if (n < n_rows) {
+          const int tq = n / G, hh = n - tq * G;
+          const float2 ml = blk_ml[n];
+          const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+          out[row * DD_D + d] = __float2bfloat16_rn(ml.y > 0.f ? ob[n] / ml.y : 0.f);
+          if (out_lse && d == 0) out_lse[row] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");        // the staging arrays are rewritten by the next segment
+      continue;
+    }
+    {
+      const int part = (int)blockIdx.x - b_first;
+      float* po = part_o + ((bg * max_parts + part) * AS_ROWS) * DD_D;
+#pragma unroll
+      for (int n = 0; n < AS_ROWS; ++n) po[n * DD_D + d] = ob[n];
+      if (d < AS_ROWS) part_ml[(bg * max_parts + part) * AS_ROWS + d] = blk_ml[d];
+      __threadfence();
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (threadIdx.x == 0) {
+      const unsigned prev = atomicAdd(&ticket[bg], 1u);
+      sm_last = (prev == (unsigned)(n_parts - 1));
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (sm_last) {
+      // ---- the last block of the unit to arrive merges the partials
+      __threadfence();
+      if (threadIdx.x == 0) ticket[bg] = 0u;           // ready for the next launch
+      float2* sm_lm = &sm_ml[0][0];                    // reused: [row] -> (max, sum)
+      float* sm_sc = &sm_o[0][0][0];                   // reused: [part][row] scale, n_parts <= AS_MAX_PARTS
+      for (int n = warp; n < AS_ROWS; n += AS_CONSUMERS) {
+        const float2* pml = part_ml + bg * max_parts * AS_ROWS + n;
+        float ms[AS_MAX_PARTS / 32], ls[AS_MAX_PARTS / 32];
+        float M = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < AS_MAX_PARTS / 32; ++i) {
+          const int sp = lane + 32 * i;
+          ms[i] = sp < n_parts ? __ldcg(&pml[sp * AS_ROWS].x) : -INFINITY;
+          ls[i] = sp < n_parts ? __ldcg(&pml[sp * AS_ROWS].y) : 0.f;
+          M = fmaxf(M, ms[i]);
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+        float L = 0.f;
+#pragma unroll
+        for (int i = 0; i < AS_MAX_PARTS / 32; ++i) {
+          const int sp = lane + 32 * i;
+          const float sc = (ms[i] == -INFINITY) ? 0.f : exp2f(ms[i] - M);
+          if (sp < n_parts) sm_sc[sp * AS_ROWS + n] = sc;
+          L += ls[i] * sc;
+        }
+#pragma unroll
+        for (int off = 16; off; off >>= 1) L += __shfl_xor_sync(0xffffffffu, L, off);
+        if (lane == 0) sm_lm[n] = make_float2(M, L);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      float a[AS_ROWS];
+#pragma unroll
+      for (int n = 0; n < AS_ROWS; ++n) a[n] = 0.f;
+      const float* po = part_o + bg * max_parts * AS_ROWS * DD_D + d;
+#pragma unroll 4
+      for (int sp = 0; sp < n_parts; ++sp) {
+#pragma unroll
+        for (int n = 0; n < AS_ROWS; ++n) a[n] += __ldcg(po + (sp * AS_ROWS + n) * DD_D) * sm_sc[sp * AS_ROWS + n];
+      }
+#pragma unroll
+      for (int n = 0; n < AS_ROWS; ++n) {
+        if (n < n_rows) {
+          const float2 ml = sm_lm[n];
+          const int tq = n / G, hh = n - tq * G;
+          const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
+          out[row * DD_D + d] = __float2bfloat16_rn(ml.y > 0.f ? a[n] / ml.y : 0.f);
+          if (out_lse && d == 0) out_lse[row] = (ml.x + log2f(ml.y)) * 0.6931471805599453f;
+        }
+      }
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");          // the staging arrays are rewritten by the next segment
+  }
+  if (PROBE && probe_acc == 0x9E3779B9u) sink[0] = probe_acc;   // keeps the loads alive; practically never true
+  if (threadIdx.x == 0 && *abort_p) dd_report(err_word, DD_ERR_WAIT_EXPIRED, 3);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+// Blocks, pages per block and partials per unit for a configuration: two blocks per SM when there is enough work
+// (at least eight pages per block), and never more than AS_MAX_PARTS blocks per unit.
+void dd_attn_stream_geometry(const dd_config* c, int sm_count, int* n_blocks, int* ppb_out, int* max_parts_out) {
+  const long long total = (long long)c->batch * c->n_kv_heads * c->k_pages;
+  long long nb = 2LL * sm_count;
+  if (nb > (total + 7) / 8) nb = (total + 7) / 8;
+  if (nb < 1) nb = 1;
+  long long ppb = (total + nb - 1) / nb;
+  while ((c->k_pages - 1) / ppb + 2 > AS_MAX_PARTS) ++ppb;
+  nb = (total + ppb - 1) / ppb;
+  *n_blocks = (int)nb;
+  *ppb_out = (int)ppb;
+  *max_parts_out = (int)((c->k_pages - 1) / ppb + 2);
+}
+
+typedef CUresult (*dd_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of one ring slot seen as [rows = B * Hkv * 2 * k * T][128 channels] bf16, boxes of 16 rows x 64 channels
+// with the 128-byte swizzle. Returns DD_OK, or an error when the driver entry point is missing or refuses the map.
+int dd_attn_stream_make_map(dd_ctx* ctx, const void* slot, void* map_out) {
+  static dd_encode_tiled_fn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+      cudaGetLastError();
+      return dd_fail(ctx, DD_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    }
+    encode = (dd_encode_tiled_fn)fn;
+  }
+  const dd_config& c = ctx->cfg;
+  const cuuint64_t dims[2] = {(cuuint64_t)DD_D, (cuuint64_t)c.batch * c.n_kv_heads * 2 * c.k_pages * DD_T};
+  const cuuint64_t strides[1] = {(cuuint64_t)DD_ROW_BYTES};
+  const cuuint32_t box[2] = {64, (cuuint32_t)DD_T};
+  const cuuint32_t elem[2] = {1, 1};
+  const CUresult r = encode((CUtensorMap*)map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(slot), dims, strides,
+                            box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return dd_fail(ctx, DD_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return DD_OK;
+}
+
+int dd_attn_stream_setup(dd_ctx* ctx) {
+  DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_attn_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AS_SMEM_BYTES));
+  DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_attn_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AS_SMEM_BYTES));
+  dd_attn_stream_geometry(&ctx->cfg, ctx->sm_count, &ctx->as_blocks, &ctx->as_ppb, &ctx->as_max_parts);
+  for (int s = 0; s < ctx->cfg.ring_depth; ++s) {
+    const int rc = dd_attn_stream_make_map(ctx, ctx->ring + (size_t)s * ctx->slot_bytes, &ctx->as_tmap[s]);
+    if (rc != DD_OK) return rc;
+  }
+  return DD_OK;
+}
+
+int dd_launch_attn_stream(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len, void* out,
+                          float* out_lse, cudaStream_t st, const void* k_new, const void* v_new, bool probe) {
+  const dd_config& c = ctx->cfg;
+  const int total = c.batch * c.n_kv_heads * c.k_pages;
+  const CUtensorMap& map = *reinterpret_cast<const CUtensorMap*>(&ctx->as_tmap[slot]);
+  if (probe)
+    dd_attn_stream_kernel<true><<<ctx->as_blocks, AS_THREADS, AS_SMEM_BYTES, st>>>(
+        map, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, c.n_kv_heads, ctx->G, c.n_q_tokens,
+        c.k_pages, total, ctx->as_ppb, ctx->as_max_parts, nullptr, nullptr, ctx->err_word, ctx->bulk_wait_ns,
+        ctx->attn_ticket + c.batch * c.n_kv_heads);
+  else
+    dd_attn_stream_kernel<false><<<ctx->as_blocks, AS_THREADS, AS_SMEM_BYTES, st>>>(
+        map, (const __nv_bfloat16*)q, idx, ctx_len, (__nv_bfloat16*)out, out_lse, ctx->attn_part_o, ctx->attn_part_ml,
+        ctx->attn_ticket, c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, total, ctx->as_ppb, ctx->as_max_parts,
+        (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, ctx->err_word, ctx->bulk_wait_ns, nullptr);
+  DD_CUDA_TRY(ctx, cudaGetLastError());
+  return DD_OK;
+}

@@ -31,10 +31,10 @@ def test_binding_lists_the_same_entry_points_and_error_strings():
     assert binding.lib.dd_strerror(0) == b"ok"
     assert binding.lib.dd_strerror(binding.DD_ERR_NOT_PINNED) == b"host memory is not page-locked"
     # size queries and configuration checks run on the host
-    cfg = binding.DDConfig(32, 8, 32, 8, 128, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0)
+    cfg = binding.DDConfig(32, 8, 32, 8, 128, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0, 0)
     assert binding.lib.dd_slot_bytes(ctypes.byref(cfg)) == 64 << 20
     assert binding.lib.dd_ring_bytes(ctypes.byref(cfg)) == 128 << 20
-    bad = binding.DDConfig(32, 8, 32, 8, 64, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0)
+    bad = binding.DDConfig(32, 8, 32, 8, 64, 16, 2048, 128, 0, 2, 2, 0, 0, 0, 0, None, None, None, 0, 0, 0, None, None, 0, 0, 0)
     assert binding.lib.dd_slot_bytes(ctypes.byref(bad)) == 0
     h = ctypes.c_void_p()
     assert binding.lib.dd_create(ctypes.byref(bad), ctypes.byref(h)) == binding.DD_ERR_INVALID_ARG

@@ -23,6 +23,12 @@ def dd():
     return binding
 
 
+@pytest.fixture(params=["stream", "split"])
+def attn_mode(request, dd):
+    """Both attention kernels serve the same entry points."""
+    return dd.DD_ATTN_STREAM if request.param == "stream" else dd.DD_ATTN_SPLIT
+
+
 def _layer_store(w, layer, pinned=True):
     """One layer of the host store [B, Hkv, P, 2, T, d] bf16 (pinned) from the seeded generator."""
     kv = torch.stack([wl.kv_slab(w, layer, b) for b in range(w.batch)])
@@ -201,7 +207,7 @@ def test_gather_rejects_pageable_memory_and_clamps_bad_indices(dd):
     c.close()
 
 
-def _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed, G=4, sharp=1.0):
+def _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed, G=4, sharp=1.0, attn_mode=0):
     Hq = HKV * G
     g = torch.Generator().manual_seed(seed)
     kv = torch.randn(B, HKV, P, 2, T, D, generator=g).to(torch.bfloat16).pin_memory()
@@ -217,7 +223,8 @@ def _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed, G=4, sharp=1.0):
             s = sorted(set(idx[b, h].tolist()))
             fill = [p for p in range(last + 1) if p not in s]
             idx[b, h] = torch.tensor(sorted(s + fill[:k - len(s)]), dtype=torch.int32)
-    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_q_tokens=Tq, attn_splits=splits)
+    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_q_tokens=Tq, attn_splits=splits,
+                   attn_mode=attn_mode)
     c.gather_kv_from_host(kv, idx.cuda(), None, 0)
     out = torch.full((B, Tq, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
     lse = torch.zeros((B, Tq, Hq), dtype=torch.float32, device="cuda")
@@ -238,15 +245,22 @@ def _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed, G=4, sharp=1.0):
     (2, 64, 3, [1024, 1000], 1, 3),                # fewer pages than warps; single query token
     (1, 40, 40, [633], 2, 7),                      # full budget, partial last page
 ])
-def test_attention_matches_oracle(dd, B, P, k, ctx_len, Tq, splits):
-    _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed=B * 1000 + k)
+def test_attention_matches_oracle(dd, attn_mode, B, P, k, ctx_len, Tq, splits):
+    _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed=B * 1000 + k, attn_mode=attn_mode)
 
 
-def test_attention_sharp_queries_and_other_group_sizes(dd):
-    _attn_case(dd, 2, 128, 32, [2048, 2040], 2, 0, seed=1, sharp=4.0)     # peaked soft-max
-    _attn_case(dd, 2, 128, 32, [2048, 2040], 2, 0, seed=2, G=2)
-    _attn_case(dd, 2, 128, 32, [2048, 2040], 1, 4, seed=3, G=8)
-    _attn_case(dd, 1, 128, 32, [2048], 2, 2, seed=4, G=1)
+def test_attention_sharp_queries_and_other_group_sizes(dd, attn_mode):
+    _attn_case(dd, 2, 128, 32, [2048, 2040], 2, 0, seed=1, sharp=4.0, attn_mode=attn_mode)     # peaked soft-max
+    _attn_case(dd, 2, 128, 32, [2048, 2040], 2, 0, seed=2, G=2, attn_mode=attn_mode)
+    _attn_case(dd, 2, 128, 32, [2048, 2040], 1, 4, seed=3, G=8, attn_mode=attn_mode)
+    _attn_case(dd, 1, 128, 32, [2048], 2, 2, seed=4, G=1, attn_mode=attn_mode)
+
+
+def test_streaming_attention_when_blocks_cut_units_at_every_offset(dd):
+    """Shapes whose flat page list is cut into per-block runs that start and end inside units, cover several whole
+    units, or hold fewer pages than consumer warps: many requests with few pages, one request with many."""
+    for B, P, k, seed in [(16, 40, 5, 1), (9, 64, 7, 2), (1, 4096, 1200, 3), (5, 200, 66, 4), (32, 64, 64, 5)]:
+        _attn_case(dd, B, P, k, [P * 16 - (3 * b) % 15 for b in range(B)], 2, 0, seed=seed, attn_mode=dd.DD_ATTN_STREAM)
 
 
 def test_full_budget_equals_dense_attention(dd):
@@ -283,7 +297,7 @@ def test_full_budget_equals_dense_attention(dd):
     (2, 64, 8, [1024, 1001], 1, 2, 8),             # one query token: it sees only its own new entry
     (3, 300, 128, [4800, 4799, 2049], 2, 0, 2),
 ])
-def test_attention_with_causal_tail_matches_oracle(dd, B, P, k, ctx_len, Tq, splits, G):
+def test_attention_with_causal_tail_matches_oracle(dd, attn_mode, B, P, k, ctx_len, Tq, splits, G):
     Hq = HKV * G
     g = torch.Generator().manual_seed(B * 77 + k)
     kv = torch.randn(B, HKV, P, 2, T, D, generator=g).to(torch.bfloat16).pin_memory()
@@ -298,7 +312,8 @@ def test_attention_with_causal_tail_matches_oracle(dd, B, P, k, ctx_len, Tq, spl
         for h in range(HKV):
             s = torch.randperm(last, generator=g)[:k - 1].tolist() + [last]
             idx[b, h] = torch.tensor(sorted(s), dtype=torch.int32)
-    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_q_tokens=Tq, attn_splits=splits)
+    c = dd.Context(n_layers=1, batch=B, max_pages=P, k_pages=k, n_q_heads=Hq, n_q_tokens=Tq, attn_splits=splits,
+                   attn_mode=attn_mode)
     c.gather_kv_from_host(kv, idx.cuda(), None, 0)
     out = torch.full((B, Tq, Hq, D), 7.0, dtype=torch.bfloat16, device="cuda")
     lse = torch.zeros((B, Tq, Hq), dtype=torch.float32, device="cuda")

@@ -95,6 +95,25 @@ def test_chain_matches_oracle_and_is_invariant_to_ring_depth_and_engine(dd):
             assert np.array_equal(i2, idxs)
 
 
+def test_chain_with_the_streaming_attention_kernel(dd):
+    """The pipelined step with the TMA-fed attention kernel: same index sets, outputs equal to the split-KV
+    kernel's up to rounding (the two merge partial results in different orders) and within tolerance of the oracle."""
+    S = 3
+    w = wl.small(wl.CONFIGS[4], n_layers=3, batch=2, ctx=16 * 90, budget=16 * 12, recent_window=32)
+    inp = _inputs(w, S)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    want, want_idx = _run(dd, w, S, inp, depth=2)
+    for depth in (2, 3):
+        got, got_idx = _run(dd, w, S, inp, depth=depth, ctx_kw=dict(attn_mode=dd.DD_ATTN_STREAM))
+        assert np.array_equal(got_idx, want_idx)
+        assert np.abs(f32(got) - f32(want)).max() <= 2e-2
+        for t in range(S):
+            for l in range(w.n_layers):
+                slot = orc.gather_kv(f32(store[l]), got_idx[t, l])
+                ref, _ = orc.sparse_decode_attn(f32(q_steps[t, l]), slot, got_idx[t, l], ctx_len.numpy(), T)
+                check_attention(got[t, l], ref)
+
+
 def test_single_layer_model_with_a_deeper_ring(dd):
     """Config 1's shape: one layer, two slots; the next step's gather is released by this step's selection."""
     S = 4
