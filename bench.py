@@ -146,12 +146,17 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def config_dict(w, **extra):
-    """The workload description both arms print."""
+L2_NOTE = ("inputs larger than L2: each layer streams its own landmarks and freshly gathered pages; the host store is "
+           "never cached")
+
+
+def config_dict(w, n_ranks=1, **extra):
+    """The workload description; both arms print exactly the same dictionary."""
     d = {"workload": w.name, "batch": w.batch, "ctx": w.ctx, "budget": w.budget, "layers": w.n_layers,
          "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim, "page_tokens": w.page_tokens,
          "forced_recent_pages": w.forced_recent_pages, "config_steps": w.steps,
-         "generator": {k: v for k, v in w.params().items() if k in GEN_KEYS}}
+         "generator": {k: v for k, v in w.params().items() if k in GEN_KEYS},
+         "parallelism": "replicas only" if n_ranks > 1 else "single GPU", "l2": L2_NOTE}
     d.update(extra)
     return d
 
@@ -261,7 +266,8 @@ def run_reference(args):
             "steps": len(times), "warmup": done_warm, "ms_per_step": ms, "extrapolated_from_layers": 1,
             "measured_ms_per_layer": per_layer * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_dict(w, parallelism="host cores only"),
+            "config": config_dict(w, n_ranks=args.gpus),
+            "engine": {"what": "CPU oracle on the host cores (numpy, fp64); no GPU work"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                              "cpu_seconds_over_wall_seconds": cpu / sum(times), "host_cores": len(os.sched_getaffinity(0))},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -639,14 +645,10 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": config_dict(
-            w, ring_depth=args.ring_depth, ragged_contexts=args.ragged, select_stream=not args.no_select_stream,
-            landmark_chunk_tokens=args.landmark_chunk or w.page_tokens, gather_mode=args.gather_mode,
-            attn_mode=args.attn_mode,
-            host_store_gib=store.host_bytes / 2**30, phys_layers=store.n_phys,
-            parallelism="replicas only" if world > 1 else "single GPU",
-            l2="inputs larger than L2: each layer streams its own landmarks and freshly gathered pages; the host "
-               "store is never cached"),
+        "config": config_dict(w, n_ranks=world),
+        "engine": {"ring_depth": args.ring_depth, "ragged_contexts": args.ragged, "select_stream": not args.no_select_stream,
+                   "landmark_chunk_tokens": args.landmark_chunk or w.page_tokens, "gather_mode": args.gather_mode,
+                   "attn_mode": args.attn_mode, "host_store_gib": store.host_bytes / 2**30, "phys_layers": store.n_phys},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": q_bytes + L * gather_bytes,
                 "d2h_bytes_per_step": o_bytes,
                 "note": "dd_decode_step_host: queries from pinned host memory and outputs back to it every step, the host "
@@ -764,7 +766,8 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
 
     def timed(stream, fn, pre=None):
         """Average device time of fn over `reps` launches enqueued back to back on `stream` (no host
-        synchronisation in between, as in the pipeline); `pre` runs before every launch and its own cost,
+        synchronisation in between, as in the pipeline; the stream is kept busy while the host enqueues, so
+        that host launch cost is not in the number); `pre` runs before every launch and its own cost,
         measured the same way, is subtracted."""
         def batch(with_fn):
             for i in range(3):
@@ -774,7 +777,9 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
                     fn(i)
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
+            with torch.cuda.stream(stream):
+                torch.cuda._sleep(3_000_000)       # ~1.5 ms of device idle-spin: the host queues the launches ahead,
+            e0.record(stream)                      # so the events bracket device time, not host enqueue time
             for i in range(reps):
                 if pre:
                     pre(i)
