@@ -64,11 +64,12 @@ int dd_gather_stats(dd_ctx* ctx, unsigned long long* out, int reset);
 
 /* ---- test hooks ------------------------------------------------------------------------------------- */
 
-/* Limit of the bounded device-side waits of the bulk gather engine (default 2 s), and a way to make one run
- * out without faulting anything: with inflate_first_stage != 0 the first stage of block 0 expects 16 bytes
- * more than its copy delivers, so its wait can never complete; the copy itself lands normally, the wait gives
- * up after wait_seconds, the block waits (bounded) for its other copies in flight and returns, and the device
- * error word reports DD_ERR_WAIT_EXPIRED. For tests of that error path only. */
+/* Limit of the bounded device-side waits (the mbarrier waits of the bulk gather engine and of the streaming
+ * attention kernel; default 2 s), and a way to make one run out without faulting anything: with
+ * inflate_first_stage != 0 the first stage of block 0 of the bulk gather expects 16 bytes more than its copy
+ * delivers, so its wait can never complete; the copy itself lands normally, the wait gives up after wait_seconds,
+ * the block waits (bounded) for its other copies in flight and returns, and the device error word reports
+ * DD_ERR_WAIT_EXPIRED. For tests of that error path only. */
 int dd_set_bulk_wait(dd_ctx* ctx, double wait_seconds, int inflate_first_stage);
 
 /* The cluster-size search of the fused selection kernel with the device queries replaced by a callback, so that
