@@ -777,9 +777,12 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
                     fn(i)
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            with torch.cuda.stream(stream):
-                torch.cuda._sleep(3_000_000)       # ~1.5 ms of device idle-spin: the host queues the launches ahead,
-            e0.record(stream)                      # so the events bracket device time, not host enqueue time
+            try:                                   # ~1.5 ms of device idle-spin: the host queues the launches ahead,
+                with torch.cuda.stream(stream):    # so the events bracket device time, not host enqueue time
+                    torch.cuda._sleep(3_000_000)
+            except Exception:
+                pass
+            e0.record(stream)
             for i in range(reps):
                 if pre:
                     pre(i)
