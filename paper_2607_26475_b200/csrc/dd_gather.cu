@@ -249,7 +249,7 @@ int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev,
                             const int* n_pages_h, const int* n_pages_dev, char* slot, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
   const int Hkv = c.n_kv_heads, P = c.max_pages, k = c.k_pages;
-  const int units = c.batch * Hkv, total = units * k;
+  const int units = c.batch * Hkv;
   const int Bp = ctx->stage_block, min_run = ctx->stage_min_run;
   const int li = (int)(ctx->list_next % DD_STAGE_LISTS);
   if (ctx->list_used[li]) {
@@ -343,7 +343,6 @@ int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev,
   ctx->gstats[3] += sel_staged;
   ctx->gstats[4] += (unsigned long long)n_strag;
   ctx->gstats[6] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t0).count();
-  (void)total;
   return DD_OK;
 }
 
