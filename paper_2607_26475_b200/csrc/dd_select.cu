@@ -517,14 +517,26 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       // acc[0], acc[1]: row gl, heads 2t, 2t+1; acc[2], acc[3]: row gl + 8
       const int r0 = tile * 16 + gl, r1 = r0 + 8;
       const bool ok0 = r0 < n_local_rows, ok1 = r1 < n_local_rows;
+      if (G == 4) {
+        // one 16-byte store per row instead of four 4-byte ones: lanes t = 0 and t = 1 of a row group swap halves,
+        // t = 0 then holds all four heads of row gl, t = 1 those of row gl + 8
+        const float a0 = (acc[0] + acc2[0]) * scale, a1 = (acc[1] + acc2[1]) * scale;      // row gl,     heads 2t, 2t+1
+        const float b0 = (acc[2] + acc2[2]) * scale, b1 = (acc[3] + acc2[3]) * scale;      // row gl + 8, heads 2t, 2t+1
+        const float x0 = __shfl_xor_sync(0xffffffffu, t == 0 ? b0 : a0, 1);
+        const float x1 = __shfl_xor_sync(0xffffffffu, t == 0 ? b1 : a1, 1);
+        if (t == 0 && ok0) *reinterpret_cast<float4*>(s_sm + (size_t)r0 * 4) = make_float4(a0, a1, x0, x1);
+        if (t == 1 && ok1) *reinterpret_cast<float4*>(s_sm + (size_t)r1 * 4) = make_float4(x0, x1, b0, b1);
+      }
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
         const int h = 2 * t + c;
         if (h < G && ok0) {
           const float v0 = (acc[c] + acc2[c]) * scale;
           const float v1 = ok1 ? (acc[2 + c] + acc2[2 + c]) * scale : v0;
-          s_sm[(size_t)r0 * G + h] = v0;
-          if (ok1) s_sm[(size_t)r1 * G + h] = v1;
+          if (G != 4) {
+            s_sm[(size_t)r0 * G + h] = v0;
+            if (ok1) s_sm[(size_t)r1 * G + h] = v1;
+          }
           const float vmax = fmaxf(v0, v1);
           mx_run[c] = fmaxf(mx_run[c], vmax);
           mn_run[c] = fminf(mn_run[c], fminf(v0, v1));
@@ -650,21 +662,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
     for (int h = 0; h < 8; ++h) lse[h] = h < G ? lse_s[h] : 0.f;
     const int width = hi_bits < RADIX_BITS ? hi_bits : RADIX_BITS;
     const int shift = hi_bits - width;
-    const bool quad = G == 4 && R == 1;          // the common shape: one 16-byte read per page
-    for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
-      float c = -INFINITY;
-      if (quad) {
-        const float4 v = *reinterpret_cast<const float4*>(s_sm + (size_t)pl * 4);
-        c = fmaxf(fmaxf(v.x - lse[0], v.y - lse[1]), fmaxf(v.z - lse[2], v.w - lse[3]));
-      } else {
-        for (int r = 0; r < R; ++r) {
-          if (pl * R + r < n_local_rows) {
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
-              if (h < G) c = fmaxf(c, s_sm[((size_t)pl * R + r) * G + h] - lse[h]);
-          }
-        }
-      }
+    auto finish = [&](int pl, float c) {
       const int p = p_lo + pl;
       if (out_scores) out_scores[bg * P + p] = expf(c);
       uint32_t key = dd_orderable(c);
@@ -672,6 +670,35 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       if (p >= n_free) key = 0xFFFFFFFFu;
       else if (width > 0) atomicAdd(&hist[(key - klo) >> shift], 1u);
       keys[pl] = key;
+    };
+    if (G == 4 && R == 1) {
+      // the common shape: one 16-byte read per page, four pages per thread in flight (the logits may sit in L2)
+      for (int base = tid; base < n_local; base += 4 * SEL_THREADS) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int pl = base + u * SEL_THREADS;
+          v[u] = pl < n_local ? *reinterpret_cast<const float4*>(s_sm + (size_t)pl * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int pl = base + u * SEL_THREADS;
+          if (pl < n_local)
+            finish(pl, fmaxf(fmaxf(v[u].x - lse[0], v[u].y - lse[1]), fmaxf(v[u].z - lse[2], v[u].w - lse[3])));
+        }
+      }
+    } else {
+      for (int pl = tid; pl < n_local; pl += SEL_THREADS) {
+        float c = -INFINITY;
+        for (int r = 0; r < R; ++r) {
+          if (pl * R + r < n_local_rows) {
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+              if (h < G) c = fmaxf(c, s_sm[((size_t)pl * R + r) * G + h] - lse[h]);
+          }
+        }
+        finish(pl, c);
+      }
     }
   }
 
@@ -681,6 +708,8 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   unsigned long long prefix = 0;
   unsigned k_rem = (unsigned)k_free;
   int shift = hi_bits;                           // bits below the resolved prefix
+  unsigned above_acc = 0;                        // this thread's share of the local keys above the chosen bins
+  unsigned eq_local = (unsigned)n_free_local;    // local keys equal to the threshold when the digits resolve it exactly
   if (k_free > 0) {
     for (int pass = 0; shift > 0; ++pass) {
       const int width = shift < RADIX_BITS ? shift : RADIX_BITS;
@@ -726,45 +755,35 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
       prefix = (prefix << width) | bin;
       k_rem -= ab;                                // keys in higher bins are all selected
       shift = nshift;
+#pragma unroll
+      for (int jb = 0; jb < 8; ++jb) {            // local keys in higher bins of this pass, counted from the histogram
+        const unsigned b8 = RADIX_BINS - 1 - 8 * tid - jb;
+        if (b8 > bin) above_acc += h[b8];
+      }
+      eq_local = h[bin];
       __syncthreads();                            // sh_grp, sh_above and cnt8 are rewritten by the next pass
       if (bin_cnt <= (unsigned)SEL_CAND_MAX) break;
     }
   }
 
-  // ---- E. publish what the peers need to finish: how many local pages are certainly selected, and the local keys
-  // that share the prefix (listed when digits remain, only counted when the prefix is the whole key)
+  // ---- E. publish what the peers need to finish: how many local pages are certainly selected (forced pages and
+  // the keys above the chosen bins, already counted from the histograms), and the local keys that share the prefix
+  // (listed when digits remain, only counted when the prefix is the whole key)
   {
-    unsigned n_above = 0, n_eq = 0;
-    for (int base = warp * 32; base < n_local; base += SEL_THREADS) {
-      const int pl = base + lane;
-      bool ab = false, eq = false;
-      uint32_t key = 0;
-      if (pl < n_local) {
-        key = keys[pl];
-        if (p_lo + pl >= n_free) ab = true;
-        else if (k_free > 0) {
-          const unsigned long long dg = (unsigned long long)(key - klo) >> shift;
-          ab = dg > prefix;
-          eq = dg == prefix;
-        }
-      }
-      n_above += __popc(__ballot_sync(0xffffffffu, ab));
-      if (shift > 0) {
-        const unsigned be = __ballot_sync(0xffffffffu, eq);
-        unsigned base_slot = 0;
-        if (lane == 0 && be) base_slot = atomicAdd(&pub.cand_n, (unsigned)__popc(be));
-        base_slot = __shfl_sync(0xffffffffu, base_slot, 0);
-        if (eq) {
-          const unsigned slot = base_slot + __popc(be & ((1u << lane) - 1u));
+    above_acc = __reduce_add_sync(0xffffffffu, above_acc);
+    if (lane == 0 && above_acc) atomicAdd(&pub.above, above_acc);
+    if (tid == 0) {
+      atomicAdd(&pub.above, (unsigned)(n_local - n_free_local));        // forced pages of this block
+      if (k_free > 0 && shift == 0) pub.eq = eq_local;
+    }
+    if (k_free > 0 && shift > 0) {
+      for (int pl = tid; pl < n_free_local; pl += SEL_THREADS) {
+        const uint32_t key = keys[pl];
+        if (((unsigned long long)(key - klo) >> shift) == prefix) {
+          const unsigned slot = atomicAdd(&pub.cand_n, 1u);
           if (slot < (unsigned)SEL_CAND_MAX) pub.cand[slot] = key;
         }
-      } else {
-        n_eq += __popc(__ballot_sync(0xffffffffu, eq));
       }
-    }
-    if (lane == 0) {
-      if (n_above) atomicAdd(&pub.above, n_above);
-      if (n_eq) atomicAdd(&pub.eq, n_eq);
     }
   }
   dd_cluster_sync();
