@@ -705,7 +705,8 @@ def run_gpu(args):
                 "hidden_fraction_target_0.9_met": bool(1.0 - (us_layer - t_c) / t_g >= 0.9),
                 "overlap_efficiency": (t_c + t_g - us_layer) / min(t_c, t_g),
                 "overlap_efficiency_is": "(compute + gather - layer time) / min(compute, gather): how much of the "
-                                         "shorter of the two ran under the other; NOT the hidden fraction of the transfer"})
+                                         "shorter of the two ran under the other; NOT the hidden fraction of the transfer (a value a few percent "
+                                         "above 1 is timing noise: the gather alone and the pipelined layer differ by < 0.3%)"})
             line["roofline_kernels"] = st.pop("roofline_kernels")
     ctx.sync()
     extras = rank == 0 and world == 1 and not args.no_extras and not args.correct_misses
@@ -764,12 +765,13 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     tmp_idx = torch.empty_like(idx[0])
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
-    def timed(stream, fn, pre=None):
+    def timed(stream, fn, pre=None, ahead=True):
         """Average device time of fn over `reps` launches enqueued back to back on `stream` (no host
         synchronisation in between, as in the pipeline; the stream is kept busy while the host enqueues, so
         that host launch cost is not in the number); `pre` runs before every launch and its own cost,
         measured the same way, is subtracted."""
         def batch(with_fn):
+            spin = ahead
             for i in range(3):
                 if pre:
                     pre(i)
@@ -778,8 +780,9 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             try:                                   # ~1.5 ms of device idle-spin: the host queues the launches ahead,
-                with torch.cuda.stream(stream):    # so the events bracket device time, not host enqueue time
-                    torch.cuda._sleep(3_000_000)
+                if spin:                           # so the events bracket device time, not host enqueue time
+                    with torch.cuda.stream(stream):
+                        torch.cuda._sleep(3_000_000)
             except Exception:
                 pass
             e0.record(stream)
@@ -797,7 +800,7 @@ def stage_timings(torch, dd, ctx, store, w, q_dev, outs, hbm_peak, link_peak, ar
     sel_us = timed(cs, lambda i: ctx.select_topk_chunked(q_dev[i % q_dev.shape[0], i % L], 1, store.landmarks[i % L],
                                                          store.n_pages_dev, store.ctx_len_dev, tmp_idx, None, stream=cs))
     gat_us = timed(xs, lambda i: ctx.gather_kv_from_host(store.kv[i % L], idx[i % L], store.n_pages_dev,
-                                                         i % args.ring_depth, stream=xs))
+                                                         i % args.ring_depth, stream=xs), ahead=False)   # milliseconds each
     ctx.gather_kv_from_host(store.kv[0], idx[0], store.n_pages_dev, 0, stream=cs)
 
     def flush_l2(i):
