@@ -64,6 +64,20 @@ int dd_gather_stats(dd_ctx* ctx, unsigned long long* out, int reset);
 
 /* ---- test hooks ------------------------------------------------------------------------------------- */
 
+/* The host's part of the staged gather without any CUDA call, so that it can be tested without a GPU. From the index
+ * set idx (host int32 [B][Hkv][k]) it forms
+ *   copies      [3 * n_copies] (source page = unit * P + page, first staging page, pages): runs of adjacent selected
+ *               pages of at least min_run pages, or, with block_pages > 0, every aligned block of that many pages that
+ *               holds a selected page (adjacent blocks merged into one copy)
+ *   map         [n_staged] staged page -> slot item (unit * k + position), -1 for a page that was only fetched along
+ *   stragglers  [n_stragglers] slot items left to the zero-copy kernel
+ * n_pages (host int32 [B]) may be NULL; an index outside [0, min(n_pages[b], P)) is clamped as on the device and the
+ * first one is reported in bad = {flag, value}. DD_ERR_INVALID_ARG when the plan does not fit staging_capacity pages or
+ * max_copies copies. */
+int dd_test_stage_plan(const int* idx, const int* n_pages, int batch, int n_kv_heads, int max_pages, int k_pages, int min_run,
+                       int block_pages, long long staging_capacity, long long* copies, long long max_copies,
+                       long long* n_copies, int* map, long long* n_staged, int* stragglers, long long* n_stragglers, int* bad);
+
 /* Limit of the bounded device-side waits (the mbarrier waits of the bulk gather engine and of the streaming
  * attention kernel; default 2 s), and a way to make one run out without faulting anything: with
  * inflate_first_stage != 0 the first stage of block 0 of the bulk gather expects 16 bytes more than its copy

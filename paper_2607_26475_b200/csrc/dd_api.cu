@@ -193,6 +193,7 @@ static void dd_free_all(dd_ctx* ctx) {
     delete[] ctx->idx_copied;
   }
   delete[] ctx->n_pages_host;
+  delete[] ctx->copy_plan;
   delete[] ctx->host_kv_orig;
   if (ctx->sel_done) {
     for (int l = 0; l < ctx->cfg.n_layers; ++l)
@@ -315,6 +316,7 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
     DD_CREATE_TRY(cudaMalloc(&ctx->staging, ctx->staging_pages * DD_PAGE_BYTES));
     DD_CREATE_TRY(cudaHostAlloc((void**)&ctx->idx_host, (size_t)2 * cfg->n_layers * total * sizeof(int), cudaHostAllocDefault));
     ctx->n_pages_host = new int[cfg->batch]();
+    ctx->copy_plan = new long long[3 * total]();
     ctx->idx_copied = new cudaEvent_t[cfg->n_layers]();
     for (int l = 0; l < cfg->n_layers; ++l)
       DD_CREATE_TRY(cudaEventCreateWithFlags(&ctx->idx_copied[l], cudaEventDisableTiming));

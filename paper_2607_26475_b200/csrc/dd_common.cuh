@@ -91,6 +91,7 @@ struct dd_ctx {
   cudaEvent_t list_free[DD_STAGE_LISTS];
   bool list_used[DD_STAGE_LISTS];
   long long list_next;
+  long long* copy_plan;    // [3 * B*Hkv*k] (source page, staging page, pages) of the gather being issued
   cudaStream_t aux_stream; // library-owned: the zero-copy kernel of the short runs, next to the copy engine
   cudaEvent_t aux_fork, aux_join;
   unsigned long long gstats[DD_GATHER_STATS_FIELDS];

@@ -245,34 +245,30 @@ int dd_wait_index_copy(dd_ctx* ctx, int layer) {
   return rc;
 }
 
-int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev, const int* idx_h, const int* idx_dev,
-                            const int* n_pages_h, const int* n_pages_dev, char* slot, cudaStream_t st) {
-  const dd_config& c = ctx->cfg;
-  const int Hkv = c.n_kv_heads, P = c.max_pages, k = c.k_pages;
-  const int units = c.batch * Hkv;
-  const int Bp = ctx->stage_block, min_run = ctx->stage_min_run;
-  const int li = (int)(ctx->list_next % DD_STAGE_LISTS);
-  if (ctx->list_used[li]) {
-    const auto tw = std::chrono::steady_clock::now();
-    const int rc = dd_wait_event(ctx, ctx->list_free[li], 30.0, "staged gather: descriptor buffer still in use");
-    ctx->gstats[5] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - tw).count();
-    if (rc != DD_OK) return rc;
-  }
-  const auto t0 = std::chrono::steady_clock::now();
-  int* map = ctx->list_host[li];
-  int* strag = map + ctx->staging_pages;
-  int n_staged = 0, n_strag = 0;
-  unsigned long long n_copies = 0, sel_staged = 0;
-  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->aux_fork, st));          // the short runs may start when the copies may
-  const char* src_base = (const char*)kv_src;
+// The host's part of the staged gather, free of any CUDA call so that it can be tested without a GPU: from the index
+// set [units][k] form the copy-engine copies (runs of adjacent selected pages of at least min_run pages, or, with
+// block_pages > 0, every aligned block of that many pages that holds a selected page, adjacent blocks merged), the map
+// staged page -> slot item (-1 for a page that was only fetched along), and the list of slot items left to the
+// zero-copy kernel. A copy is three numbers: source page (unit * P + page), first staging page, pages. Indices outside
+// [0, limit) are clamped like on the device and the first one is reported in bad[2] = {flag, value}.
+extern "C" int dd_test_stage_plan(const int* idx, const int* n_pages, int batch, int n_kv_heads, int max_pages, int k_pages,
+                                  int min_run, int block_pages, long long staging_capacity, long long* copies,
+                                  long long max_copies, long long* n_copies_out, int* map, long long* n_staged_out,
+                                  int* stragglers, long long* n_stragglers_out, int* bad) {
+  if (!idx || !copies || !map || !stragglers || !n_copies_out || !n_staged_out || !n_stragglers_out || batch < 1 ||
+      n_kv_heads < 1 || max_pages < 1 || k_pages < 1 || min_run < 1 || block_pages < 0)
+    return DD_ERR_INVALID_ARG;
+  const int Hkv = n_kv_heads, P = max_pages, k = k_pages, Bp = block_pages;
+  const int units = batch * Hkv;
+  long long n_staged = 0, n_strag = 0, n_copies = 0;
   for (int bg = 0; bg < units; ++bg) {
     int limit = P;
-    if (n_pages_h) limit = n_pages_h[bg / Hkv] < P ? n_pages_h[bg / Hkv] : P;
-    const int* row = idx_h + (size_t)bg * k;
+    if (n_pages) limit = n_pages[bg / Hkv] < P ? n_pages[bg / Hkv] : P;
+    const int* row = idx + (size_t)bg * k;
     auto page_of = [&](int j) {
       int p = row[j];
       if (p < 0 || p >= limit) {
-        if (ctx->host_err[0] == 0) { ctx->host_err[0] = DD_ERR_INDEX_RANGE; ctx->host_err[1] = p; }
+        if (bad && bad[0] == 0) { bad[0] = 1; bad[1] = p; }
         p = p < 0 ? 0 : (limit > 0 ? limit - 1 : 0);
       }
       return p;
@@ -298,39 +294,73 @@ int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev,
         page0 = p;
         n_pages_copy = jj - j;
         if (n_pages_copy < min_run) {
-          for (int x = j; x < jj; ++x) strag[n_strag++] = bg * k + x;
+          for (int x = j; x < jj; ++x) stragglers[n_strag++] = bg * k + x;
           j = jj;
           continue;
         }
       }
-      if ((size_t)n_staged + n_pages_copy > ctx->staging_pages)
-        return dd_fail(ctx, DD_ERR_INVALID_ARG, "staged gather: staging region too small (index set not ascending?)");
+      if (n_staged + n_pages_copy > staging_capacity || n_copies >= max_copies) return DD_ERR_INVALID_ARG;
       for (int x = 0; x < n_pages_copy; ++x) map[n_staged + x] = -1;
       for (int x = j; x < jj; ++x) map[n_staged + page_of(x) - page0] = bg * k + x;
-      DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->staging + (size_t)n_staged * DD_PAGE_BYTES,
-                                       src_base + ((size_t)bg * P + page0) * DD_PAGE_BYTES,
-                                       (size_t)n_pages_copy * DD_PAGE_BYTES, cudaMemcpyDefault, st));
+      copies[3 * n_copies + 0] = (long long)bg * P + page0;
+      copies[3 * n_copies + 1] = n_staged;
+      copies[3 * n_copies + 2] = n_pages_copy;
       ++n_copies;
-      sel_staged += (unsigned long long)(jj - j);
       n_staged += n_pages_copy;
       j = jj;
     }
   }
+  *n_copies_out = n_copies;
+  *n_staged_out = n_staged;
+  *n_stragglers_out = n_strag;
+  return DD_OK;
+}
+
+int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev, const int* idx_h, const int* idx_dev,
+                            const int* n_pages_h, const int* n_pages_dev, char* slot, cudaStream_t st) {
+  const dd_config& c = ctx->cfg;
+  const int Hkv = c.n_kv_heads, P = c.max_pages, k = c.k_pages;
+  const long long total = (long long)c.batch * Hkv * k;
+  const int li = (int)(ctx->list_next % DD_STAGE_LISTS);
+  if (ctx->list_used[li]) {
+    const auto tw = std::chrono::steady_clock::now();
+    const int rc = dd_wait_event(ctx, ctx->list_free[li], 30.0, "staged gather: descriptor buffer still in use");
+    ctx->gstats[5] += (unsigned long long)std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - tw).count();
+    if (rc != DD_OK) return rc;
+  }
+  const auto t0 = std::chrono::steady_clock::now();
+  int* map = ctx->list_host[li];
+  int* strag = map + ctx->staging_pages;
+  long long n_staged = 0, n_strag = 0, n_copies = 0;
+  int bad[2] = {0, 0};
+  if (dd_test_stage_plan(idx_h, n_pages_h, c.batch, Hkv, P, k, ctx->stage_min_run, ctx->stage_block,
+                         (long long)ctx->staging_pages, ctx->copy_plan, total, &n_copies, map, &n_staged, strag, &n_strag,
+                         bad) != DD_OK)
+    return dd_fail(ctx, DD_ERR_INVALID_ARG, "staged gather: staging region too small (index set not ascending?)");
+  if (bad[0] && ctx->host_err[0] == 0) { ctx->host_err[0] = DD_ERR_INDEX_RANGE; ctx->host_err[1] = bad[1]; }
+  DD_CUDA_TRY(ctx, cudaEventRecord(ctx->aux_fork, st));          // the short runs may start when the copies may
+  const char* src_base = (const char*)kv_src;
+  unsigned long long sel_staged = (unsigned long long)(total - n_strag);
+  for (long long i = 0; i < n_copies; ++i) {
+    const long long* cp = ctx->copy_plan + 3 * i;
+    DD_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->staging + (size_t)cp[1] * DD_PAGE_BYTES, src_base + (size_t)cp[0] * DD_PAGE_BYTES,
+                                     (size_t)cp[2] * DD_PAGE_BYTES, cudaMemcpyDefault, st));
+  }
   if (n_strag > 0) {
     int ctas = c.gather_ctas > 0 ? c.gather_ctas : 16;
-    const int max_ctas = (n_strag + 7) / 8;
+    const int max_ctas = (int)((n_strag + 7) / 8);
     if (ctas > max_ctas) ctas = max_ctas;
     DD_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->aux_stream, ctx->aux_fork, 0));
     dd_gather_list_kernel<<<ctas, 256, 0, ctx->aux_stream>>>((const char*)kv_dev, idx_dev, n_pages_dev,
-                                                             ctx->list_dev[li] + ctx->staging_pages, n_strag, slot, Hkv, P,
+                                                             ctx->list_dev[li] + ctx->staging_pages, (int)n_strag, slot, Hkv, P,
                                                              k, ctx->err_word);
     DD_CUDA_TRY(ctx, cudaGetLastError());
     DD_CUDA_TRY(ctx, cudaEventRecord(ctx->aux_join, ctx->aux_stream));
   }
   if (n_staged > 0) {
-    int blocks = (n_staged + 7) / 8;
+    int blocks = (int)((n_staged + 7) / 8);
     if (blocks > 4 * ctx->sm_count) blocks = 4 * ctx->sm_count;
-    dd_assemble_kernel<<<blocks, 256, 0, st>>>(ctx->staging, ctx->list_dev[li], n_staged, slot, k);
+    dd_assemble_kernel<<<blocks, 256, 0, st>>>(ctx->staging, ctx->list_dev[li], (int)n_staged, slot, k);
     DD_CUDA_TRY(ctx, cudaGetLastError());
   }
   if (n_strag > 0) DD_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->aux_join, 0));
@@ -338,7 +368,7 @@ int dd_launch_gather_staged(dd_ctx* ctx, const void* kv_src, const void* kv_dev,
   ctx->list_used[li] = true;
   ++ctx->list_next;
   ctx->gstats[0] += 1;
-  ctx->gstats[1] += n_copies;
+  ctx->gstats[1] += (unsigned long long)n_copies;
   ctx->gstats[2] += (unsigned long long)n_staged * DD_PAGE_BYTES;
   ctx->gstats[3] += sel_staged;
   ctx->gstats[4] += (unsigned long long)n_strag;
