@@ -129,3 +129,27 @@ def test_chain_with_the_staged_gather_equals_the_direct_gather(dd, depth, kw):
     a, ai = _run(dd, w1, S, inp1, depth=2)
     b, bi = _run(dd, w1, S, inp1, depth=2, mode=dd.DD_GATHER_STAGED, ctx_kw=dict(stage_min_run_pages=1))
     assert np.array_equal(raw16(a), raw16(b)) and np.array_equal(ai, bi)
+
+
+def test_whole_step_from_host_buffers_with_the_staged_gather(dd):
+    """dd_decode_step_host on a context with the staged gather: same bits as the layer-by-layer calls with the
+    direct gather, and the counters show that both the copy engine and the zero-copy kernel carried pages."""
+    S = 3
+    w = wl.small(wl.CONFIGS[2], n_layers=3, batch=2, ctx=16 * 80, budget=16 * 20)
+    inp = _inputs(w, S)
+    store, lms, ctx_len, npg, q_init, q_steps = inp
+    want, _ = _run(dd, w, S, inp, depth=2, read_idx=False)
+    c = dd.Context(n_layers=w.n_layers, batch=w.batch, max_pages=w.n_pages, k_pages=w.k_pages,
+                   gather_mode=dd.DD_GATHER_STAGED, stage_min_run_pages=2)
+    c.bind([x.cuda() for x in lms], store, npg.cuda(), ctx_len.cuda())
+    c.prime(q_init.cuda())
+    qh = q_steps.pin_memory()
+    oh = torch.zeros_like(q_steps).pin_memory()
+    for t in range(S):
+        c.decode_step_host(t, qh[t], oh[t])
+    c.sync()
+    assert c.device_error() == (0, 0)
+    assert np.array_equal(raw16(oh), raw16(want))
+    st = c.gather_stats()
+    assert st["gathers"] >= S * w.n_layers and st["pages_staged"] > 0 and st["pages_zero_copy"] > 0
+    c.close()
