@@ -74,7 +74,7 @@ typedef struct dd_config {
   int forced_recent_pages;   /* last pages of every request that are always selected; counted inside k */
   int n_q_tokens;            /* Tq: 1 or 2 */
   int ring_depth;            /* D >= 2 (2 = the two-buffer scheme) */
-  int gather_mode;           /* DD_GATHER_LOADS or DD_GATHER_BULK */
+  int gather_mode;           /* DD_GATHER_LOADS, DD_GATHER_BULK or DD_GATHER_STAGED */
   int gather_ctas;           /* thread blocks the gather may occupy; 0 = library default */
   int select_mode;           /* DD_SELECT_AUTO or DD_SELECT_TWO_KERNELS */
   int attn_splits;           /* blocks per (request, KV head) in attention, <= 64 or a multiple of 8 up to 512; 0 = automatic */
@@ -97,7 +97,9 @@ typedef struct dd_config {
 /* ---- context ------------------------------------------------------------------------------- */
 
 /* Validates the configuration, allocates events, scratch, the index tables [2][L][B][Hkv][k]
- * and (if ring_mem is NULL) the ring of D slots on the current device. */
+ * and (if ring_mem is NULL) the ring of D slots on the current device. DD_GATHER_STAGED adds a staging region of
+ * one slot's size (times stage_block_pages with over-fetch), page-locked copies of the index tables and descriptor
+ * buffers, and one library-owned stream for the zero-copy part of a gather. */
 int dd_create(const dd_config* cfg, dd_ctx** out);
 /* Waits for the context's streams (bounded, 10 s) and frees what dd_create allocated. */
 int dd_destroy(dd_ctx* ctx);
