@@ -184,6 +184,7 @@ static void dd_free_all(dd_ctx* ctx) {
     if (ctx->list_host[i]) cudaFreeHost(ctx->list_host[i]);
     if (ctx->list_free[i]) cudaEventDestroy(ctx->list_free[i]);
   }
+  if (ctx->as_fence) cudaEventDestroy(ctx->as_fence);
   if (ctx->aux_fork) cudaEventDestroy(ctx->aux_fork);
   if (ctx->aux_join) cudaEventDestroy(ctx->aux_join);
   if (ctx->aux_stream) cudaStreamDestroy(ctx->aux_stream);
@@ -335,6 +336,10 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   if (rc == DD_OK) rc = dd_gather_setup(ctx);
   ctx->attn_stream = cfg->attn_mode == DD_ATTN_STREAM;   // measured slower than the split-KV kernel: opt-in only
   if (rc == DD_OK && ctx->attn_stream) rc = dd_attn_stream_setup(ctx);
+  if (rc == DD_OK && ctx->attn_stream && cudaEventCreate(&ctx->as_fence) != cudaSuccess) {
+    snprintf(ctx->errmsg, sizeof(ctx->errmsg), "dd_create: cannot create the streaming kernel's fence event");
+    rc = DD_ERR_CUDA;
+  }
   if (rc != DD_OK) {
     memcpy(g_errmsg, ctx->errmsg, 512);
     dd_free_all(ctx);
@@ -698,6 +703,10 @@ static int dd_layer_step_body(dd_ctx* ctx, int step, int layer, const void* q, c
   DD_TRY(dd_launch_attn(ctx, q, ctx->ring + (size_t)slot * ctx->slot_bytes, attn_idx, ctx->ctx_len, out, nullptr, cs,
                         k_new, v_new));
   if (tr) DD_CUDA_TRY(ctx, cudaEventRecord(tr[2], cs));
+  // Measured: with the streaming kernel the layer period grows from 1318 to 1860 us when nothing but events
+  // without timing follow the launch, and is back at 1318 us with one timing-enabled event recorded next to it
+  // (before or after; it makes the stream take a completion timestamp). The split-KV kernel shows no such effect.
+  else if (ctx->as_fence) DD_CUDA_TRY(ctx, cudaEventRecord(ctx->as_fence, cs));
   DD_CUDA_TRY(ctx, cudaEventRecord(ctx->released[slot], cs));                        // buffer released
   ctx->released_recorded[slot] = true;
   if (!c.miss_correction && !side_select) {

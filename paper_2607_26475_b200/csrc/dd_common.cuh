@@ -29,6 +29,7 @@ struct dd_ctx {
   int attn_splits;       // resolved blocks per (request, KV head)
   int attn_cluster;      // blocks per thread-block cluster (divides attn_splits)
   int attn_stream;       // 1: the streaming attention kernel serves the context's calls, 0: the split-KV kernel
+  cudaEvent_t as_fence;  // timing-enabled event recorded behind the streaming kernel inside the layer step (see dd_api.cu)
   int as_blocks, as_ppb, as_max_parts;   // streaming kernel: grid, pages per block, partials per unit
   struct alignas(64) { unsigned char bytes[128]; } as_tmap[DD_MAX_RING];   // tensor map of every ring slot
   int sel_cluster;       // blocks per cluster of the fused selection kernel; 0 = two-kernel path
