@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
   __shared__ float2 blk_ml[ATTN_ROWS];
   __shared__ int sm_last;
 
+  dd_grid_dependency_wait();
   // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G)
   uint4 qf[4];
   if (gl < n_rows) {
@@ -409,13 +410,14 @@ static cudaError_t dd_attn_launch_raw(cudaStream_t st, int batch, int Hkv, int G
   cfg.blockDim = dim3(ATTN_THREADS);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = cluster;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
+  cudaLaunchAttribute attr[2];
+  dd_pdl_attr(&attr[0]);
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = cluster > 1 ? 1 : 0;
+  cfg.numAttrs = cluster > 1 ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, dd_attn_kernel, (const __nv_bfloat16*)q, slot, idx, ctx_len, (__nv_bfloat16*)out,
                             out_lse, part_o, part_ml, ticket, Hkv, G, Tq, k, n_splits, pps, cluster,
                             (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
@@ -448,6 +450,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_loads_only_kernel(con
   const char* vbase = kbase + (size_t)k * DD_HALF_PAGE_BYTES;
   const int p_begin = split * pages_per_split;
   const int p_end = min(k, p_begin + pages_per_split);
+  dd_grid_dependency_wait();
   unsigned int acc = 0;
   for (int j = p_begin + warp; j < p_end; j += ATTN_WARPS) {
     uint4 klo[4], khi[4], v[4][2];
@@ -468,9 +471,16 @@ int dd_launch_attn_loads_only(dd_ctx* ctx, const char* slot, cudaStream_t st) {
     return dd_launch_attn_stream(ctx, nullptr, (int)((size_t)(slot - ctx->ring) / ctx->slot_bytes), nullptr, nullptr, nullptr,
                                  nullptr, st, nullptr, nullptr, true);
   const int S = ctx->attn_splits;
-  dd_attn_loads_only_kernel<<<dim3(S, c.n_kv_heads, c.batch), ATTN_THREADS, 0, st>>>(
-      slot, c.n_kv_heads, c.k_pages, (c.k_pages + S - 1) / S, ctx->attn_ticket + c.batch * c.n_kv_heads);
-  DD_CUDA_TRY(ctx, cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(S, c.n_kv_heads, c.batch);
+  cfg.blockDim = dim3(ATTN_THREADS);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  dd_pdl_attr(&attr[0]);                         // launched the way the kernel it stands in for is
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  DD_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, dd_attn_loads_only_kernel, slot, c.n_kv_heads, c.k_pages, (c.k_pages + S - 1) / S,
+                                      ctx->attn_ticket + c.batch * c.n_kv_heads));
   return DD_OK;
 }
 

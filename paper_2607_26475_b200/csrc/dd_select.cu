@@ -467,6 +467,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_fused_kernel(
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int gl = lane >> 2, t = lane & 3;
   const size_t bg = (size_t)b * Hkv + g;
+  dd_grid_dependency_wait();
   int np = n_pages[b];
   if (np > P || np < k) {
     if (tid == 0 && rank == 0) dd_report(err_word, DD_ERR_INDEX_RANGE, np);
@@ -901,6 +902,7 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_loads_only_kernel(co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gl = lane >> 2, t = lane & 3;
   const size_t bg = (size_t)b * Hkv + g;
+  dd_grid_dependency_wait();
   const int np = min(n_pages[b], P);
   const int row_lo = rank * ppc * R, row_max = P * R - 1;
   const int n_local_rows = max(0, min(np * R, row_lo + ppc * R) - row_lo);
@@ -945,10 +947,18 @@ __global__ void __launch_bounds__(SEL_THREADS, 2) dd_select_loads_only_kernel(co
 int dd_launch_select_loads_only(dd_ctx* ctx, const void* landmarks, const int* n_pages, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
   if (ctx->sel_cluster <= 0) return dd_fail(ctx, DD_ERR_STATE, "the load-only probe follows the fused selection kernel");
-  dd_select_loads_only_kernel<<<dim3(ctx->sel_cluster, c.n_kv_heads, c.batch), SEL_THREADS, ctx->sel_smem_bytes, st>>>(
-      (const __nv_bfloat16*)landmarks, n_pages, c.max_pages, c.n_kv_heads, ctx->sel_ppc, ctx->R, ctx->sel_stages,
-      ctx->attn_ticket + c.batch * c.n_kv_heads);
-  DD_CUDA_TRY(ctx, cudaGetLastError());
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctx->sel_cluster, c.n_kv_heads, c.batch);
+  cfg.blockDim = dim3(SEL_THREADS);
+  cfg.dynamicSmemBytes = ctx->sel_smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  dd_pdl_attr(&attr[0]);                         // launched the way the kernel it stands in for is
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  DD_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, dd_select_loads_only_kernel, (const __nv_bfloat16*)landmarks, n_pages,
+                                      c.max_pages, c.n_kv_heads, ctx->sel_ppc, ctx->R, ctx->sel_stages,
+                                      ctx->attn_ticket + c.batch * c.n_kv_heads));
   return DD_OK;
 }
 
@@ -970,13 +980,14 @@ int dd_launch_select(dd_ctx* ctx, const void* q, int q_token, int q_tokens_in_te
     cfg.blockDim = dim3(SEL_THREADS);
     cfg.dynamicSmemBytes = ctx->sel_smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = ctx->sel_cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    dd_pdl_attr(&attr[1]);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     DD_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, dd_select_fused_kernel, (const __nv_bfloat16*)q,
                                         q_tokens_in_tensor * c.n_q_heads * DD_D, q_token * c.n_q_heads * DD_D,
                                         (const __nv_bfloat16*)landmarks, n_pages, out_idx, out_scores, c.max_pages, G,
