@@ -10,7 +10,7 @@ later layer on the side stream (dd_decode_layer_step). `value` counts output tok
 The headline line is the batch-8 / 32K-context workload with its own 64 decode steps. The same line carries,
 measured in the same run: the gather engines side by side (`gather_modes`, with the run-length histogram of the
 selected sets), one pass with miss correction (`miss_correction`), and compact results of the other
-workloads (`other_configs`). `--sweeps` adds a ring-depth and a gather-grid sweep.
+workloads (`other_configs`). `--sweeps` adds a ring-depth sweep, a gather-grid sweep and miss correction against the miss rate.
 
 N > 1 runs N independent replicas, one per GPU (the path has no exchange step): under torchrun as launched,
 otherwise this script starts the N ranks itself. `--impl reference` times the CPU oracle on the host cores
@@ -84,7 +84,7 @@ def parse_args():
     ap.add_argument("--no-stages", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the gather-engine comparison, the miss-correction pass and the other workloads")
-    ap.add_argument("--sweeps", action="store_true", help="add ring_depth_sweep and gather_ctas_sweep to the line")
+    ap.add_argument("--sweeps", action="store_true", help="add ring_depth_sweep, gather_ctas_sweep and miss_rate_sweep to the line")
     ap.add_argument("--cpu-stub", action="store_true",
                     help="multi-rank plumbing only: no CUDA, gloo backend, a made-up per-rank measurement (used by the tests)")
     return ap.parse_args()
@@ -528,6 +528,41 @@ def correction_pass(b, link_peak, steps=8, warm=2):
             "note": "attention runs over the set selected from the current token; counts include warm-up"}
 
 
+def miss_rate_sweep(b, link_peak, fidelities=(0.995, 0.97, 0.9, 0.8, 0.6, 0.3), steps=4, warm=2):
+    """Miss correction against the miss rate (Sec. 6.4's priority-scheduling experiment, on synthetic queries): for
+    every fidelity of the speculated query the same steps run with the missing pages on a high-priority stream of
+    their own and with the missing pages queued behind the prefetches on the copy stream (FIFO)."""
+    torch, wl, w0 = b.torch, b.wl, b.w
+    steps, warm = min(steps, b.K), min(warm, b.W)
+    keep = (b.w, b.q_dev, b.q_init)
+    out = {}
+    try:
+        for f in fidelities:
+            w = wl.small(w0, spec_fidelity=f)
+            q = torch.stack([torch.stack([wl.queries(w, t, l) for l in range(w.n_layers)]) for t in range(steps + warm)])
+            b.w, b.q_dev = w, q.cuda()
+            b.q_init = torch.stack([wl.queries(w, -1, l)[:, 1] for l in range(w.n_layers)]).cuda()
+            row = {}
+            for name, fifo in (("priority", False), ("fifo", True)):
+                ctx = b.make_ctx(correct=True, urgent_fifo=fifo)
+                b.store.bind(ctx)
+                ms, _ = b.timed(ctx, K=steps, W=warm)
+                miss = ctx.miss_stats(reset=True)
+                ctx.close()
+                rate = miss[0] / max(1, miss[1])
+                us_layer = ms / (steps * w.n_layers) * 1e3
+                link_us = w.gathered_bytes_per_layer * (1.0 + rate) / (link_peak * 1e9) * 1e6
+                row["miss_rate"] = rate
+                row[name] = {"ms_per_step": ms / steps, "us_per_layer": us_layer, "tok_s": w.batch * steps / (ms * 1e-3),
+                             "frac_of_link_roofline": link_us / us_layer}
+            out[str(f)] = row
+    finally:
+        b.w, b.q_dev, b.q_init = keep
+    out["note"] = ("spec_fidelity = correlation of a step's speculated query with the next step's current query; priority = "
+                   "missing pages on their own high-priority stream, fifo = queued behind the prefetches on the copy stream")
+    return out
+
+
 def measure_other_config(mods, n, args, rank, world, hbm_peak, link_peak):
     """A compact measurement of another workload: pipelined tok/s, e2e, per-kernel times and roofline fractions.
     The host store keeps two physical layers (logical layer l uses l mod 2; per-layer bytes, page scatter and the
@@ -718,6 +753,8 @@ def run_gpu(args):
     if rank == 0 and world == 1 and args.sweeps:
         line["ring_depth_sweep"] = sweep(b, "ring_depth", [2, 3, 4], link_peak)
         line["gather_ctas_sweep"] = sweep(b, "gather_ctas", [8, 12, 16, 24, 32], link_peak)
+        log("miss correction against the miss rate ...")
+        line["miss_rate_sweep"] = miss_rate_sweep(b, link_peak)
     b.close()
     if extras and args.config == 2 and not (args.layers or args.batch):
         del b, ctx, store
