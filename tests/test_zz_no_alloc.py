@@ -103,3 +103,44 @@ def test_static_entry_point_rejects_memory_the_device_cannot_use():
     dd.sparse_decode_attn_static(q, slot, idx, cl, out, n_splits=2)      # the device is still usable
     torch.cuda.synchronize()
     assert bool((out == 0.0).all())
+
+
+def test_static_entry_point_inside_a_cuda_graph():
+    """The call allocates nothing and is ordered by its stream only, so it can be captured: a graph that holds two
+    calls (different split counts, the second finds the first one's leftovers in the scratch array) is replayed on
+    fresh inputs written into the captured buffers and must give the eager call's bits."""
+    from paper_2607_26475_b200 import binding as dd
+    B, P, k = 2, 160, 48
+    g = torch.Generator().manual_seed(9)
+    idx = torch.stack([torch.stack([torch.randperm(P, generator=g)[:k].sort().values for _ in range(HKV)])
+                       for _ in range(B)]).to(torch.int32).cuda()
+    cl = torch.tensor([P * T, P * T - 5], dtype=torch.int32).cuda()
+    q = torch.zeros(B, 2, 32, D, dtype=torch.bfloat16, device="cuda")
+    slot = torch.zeros(B, HKV, 2, k * T, D, dtype=torch.bfloat16, device="cuda")
+    out_a, out_b = torch.zeros_like(q), torch.zeros_like(q)
+    lse_a = torch.zeros(B, 2, 32, dtype=torch.float32, device="cuda")
+    # the first call on the device looks up the scratch array: before the capture begins
+    dd.sparse_decode_attn_static(q, slot, idx, cl, out_a, lse_a, n_splits=1)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s):
+        dd.sparse_decode_attn_static(q, slot, idx, cl, out_a, lse_a, n_splits=6, stream=s)
+        dd.sparse_decode_attn_static(q, slot, idx, cl, out_b, None, n_splits=3, stream=s)
+    for rep in range(3):
+        q.copy_(torch.randn(q.shape, generator=g).to(torch.bfloat16))
+        slot.copy_(torch.randn(slot.shape, generator=g).to(torch.bfloat16))
+        out_a.fill_(7.0)
+        out_b.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        want_a, want_b = torch.zeros_like(q), torch.zeros_like(q)
+        want_lse = torch.zeros_like(lse_a)
+        dd.sparse_decode_attn_static(q, slot, idx, cl, want_a, want_lse, n_splits=6)
+        dd.sparse_decode_attn_static(q, slot, idx, cl, want_b, None, n_splits=3)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, want_a) and torch.equal(out_b, want_b) and torch.equal(lse_a, want_lse)
+        from oracle import dd_oracle as orc
+        ref, _ = orc.sparse_decode_attn(f32(q), f32(slot), idx.cpu().numpy(), cl.cpu().numpy(), T)
+        check_attention(out_a, ref)
+        check_attention(out_b, ref)
