@@ -80,11 +80,16 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
   __shared__ float sm_o[ATTN_WARPS][DD_D][ATTN_OPAD];   // per-warp O^T, [channel][row]
   __shared__ float2 sm_ml[ATTN_WARPS][ATTN_ROWS];
   __shared__ float sm_scale[ATTN_WARPS][ATTN_ROWS];
-  __shared__ float blk_o[ATTN_ROWS][DD_D];              // block result, read by the cluster's other blocks
+  // what the blocks of the cluster send each other: block r owns the channels [r*128/C, (r+1)*128/C) and receives
+  // every block's partial of them, [source block][row][channel of the slice], plus every block's (max, sum)
+  __shared__ float recv_o[ATTN_ROWS * DD_D];
+  __shared__ float2 recv_ml[ATTN_MAX_CLUSTER][ATTN_ROWS];
   __shared__ float2 blk_ml[ATTN_ROWS];
   __shared__ int sm_last;
 
   dd_grid_dependency_wait();
+  // arrives now, waits just before the first write into a peer's shared memory: by then every block has started
+  if (cluster > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   // B operand of S^T: column n = gl is query row (token n / G, head g*G + n % G)
   uint4 qf[4];
   if (gl < n_rows) {
@@ -283,25 +288,37 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
   const int n_groups = n_splits / cluster;       // clusters per (request, KV head)
   const int group = split / cluster;
   if (cluster > 1) {
-    // ---- merge the blocks of the cluster through distributed shared memory: block `rank` reduces the
-    // channels [rank*128/cluster, (rank+1)*128/cluster) of all rows over every block of the cluster
+    // ---- merge the blocks of the cluster through distributed shared memory. Every block sends the slice of its
+    // partial that block r owns into r's receive buffer (remote stores, nobody waits for an answer), one cluster
+    // barrier makes them visible, and every block reduces its slice from its own shared memory. Nothing remote is
+    // touched after the barrier, so a block may leave as soon as it is done.
     namespace cg = cooperative_groups;
     cg::cluster_group cl = cg::this_cluster();
     const int rank = (int)cl.block_rank();
-#pragma unroll
-    for (int n = 0; n < ATTN_ROWS; ++n) blk_o[n][d] = ob[n];
-    cl.sync();
     const int ch = DD_D / cluster;               // channels per block
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // pairs with the arrive at the top
+    {
+      const int r = d / ch, dd = d - r * ch;
+      float* dst = cl.map_shared_rank(recv_o, r) + (size_t)rank * ATTN_ROWS * ch + dd;
+#pragma unroll
+      for (int n = 0; n < ATTN_ROWS; ++n) dst[n * ch] = ob[n];
+      if (d < ATTN_ROWS * cluster) {
+        const int rr = d / ATTN_ROWS, n = d - rr * ATTN_ROWS;
+        *cl.map_shared_rank(&recv_ml[rank][n], rr) = blk_ml[n];
+      }
+    }
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     for (int e = threadIdx.x; e < ATTN_ROWS * ch; e += ATTN_THREADS) {
-      const int n = e / ch, dd = rank * ch + (e - n * ch);
+      const int n = e / ch, dd = e - n * ch;
       float ms[ATTN_MAX_CLUSTER], ls[ATTN_MAX_CLUSTER], os[ATTN_MAX_CLUSTER];
       float M = -INFINITY;
 #pragma unroll
       for (int r = 0; r < ATTN_MAX_CLUSTER; ++r) {
         if (r < cluster) {
-          const float2 ml = *cl.map_shared_rank(&blk_ml[n], r);
+          const float2 ml = recv_ml[r][n];
           ms[r] = ml.x; ls[r] = ml.y;
-          os[r] = *cl.map_shared_rank(&blk_o[n][dd], r);
+          os[r] = recv_o[(r * ATTN_ROWS + n) * ch + dd];
           M = fmaxf(M, ml.x);
         }
       }
@@ -314,21 +331,25 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_kernel(
           a += os[r] * sc;
         }
       }
+      const int dg = rank * ch + dd;             // channel of the head
       if (n_groups == 1) {
         if (n < n_rows) {
           const int tq = n / G, hh = n - tq * G;
           const size_t row = ((size_t)b * Tq + tq) * Hq + g * G + hh;
-          out[row * DD_D + dd] = __float2bfloat16_rn(L > 0.f ? a / L : 0.f);
-          if (out_lse && dd == 0) out_lse[row] = (M + log2f(L)) * 0.6931471805599453f;
+          out[row * DD_D + dg] = __float2bfloat16_rn(L > 0.f ? a / L : 0.f);
+          if (out_lse && dg == 0) out_lse[row] = (M + log2f(L)) * 0.6931471805599453f;
         }
       } else {
-        part_o[((bg * n_groups + group) * ATTN_ROWS + n) * DD_D + dd] = a;
-        if (dd == 0) part_ml[(bg * n_groups + group) * ATTN_ROWS + n] = make_float2(M, L);
+        part_o[((bg * n_groups + group) * ATTN_ROWS + n) * DD_D + dg] = a;
+        if (dg == 0) part_ml[(bg * n_groups + group) * ATTN_ROWS + n] = make_float2(M, L);
       }
     }
-    if (n_groups > 1) __threadfence();
-    cl.sync();                                   // nobody leaves while its shared memory may still be read
-    if (n_groups == 1 || rank != 0) return;
+    if (n_groups == 1) return;
+    // several clusters per unit: the ticket below must follow every block's partial stores
+    __threadfence();
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    if (rank != 0) return;
   } else {
     // ---- one block per cluster: publish the block's partial directly
     float* po = part_o + ((bg * n_groups + group) * ATTN_ROWS) * DD_D;
