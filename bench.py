@@ -63,7 +63,7 @@ def parse_args():
     ap.add_argument("--stage-min-run", type=int, default=0, help="staged gather: shortest run the copy engine takes (0 = 8)")
     ap.add_argument("--stage-block", type=int, default=0, help="staged gather: aligned block size in pages (0 = exact runs)")
     ap.add_argument("--attn-splits", type=int, default=0)
-    ap.add_argument("--attn-mode", default="auto", choices=["auto", "split", "stream"],
+    ap.add_argument("--attn-mode", default="auto", choices=["auto", "split", "stream", "tc"],
                     help="attention kernel: split-KV with cluster merge, or TMA-fed streaming (auto = library default)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling of small cases only)")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of small cases only)")
@@ -314,7 +314,8 @@ class Bench:
                   gather_ctas=a.gather_ctas, attn_splits=a.attn_splits, compute_stream=self.compute,
                   copy_stream=self.copy, landmark_chunk_tokens=a.landmark_chunk, select_stream=self.select,
                   stage_min_run_pages=a.stage_min_run, stage_block_pages=a.stage_block,
-                  attn_mode={"auto": dd.DD_ATTN_AUTO, "split": dd.DD_ATTN_SPLIT, "stream": dd.DD_ATTN_STREAM}[a.attn_mode])
+                  attn_mode={"auto": dd.DD_ATTN_AUTO, "split": dd.DD_ATTN_SPLIT, "stream": dd.DD_ATTN_STREAM,
+                             "tc": dd.DD_ATTN_TC}[a.attn_mode])
         if over.pop("correct", a.correct_misses):
             fifo = over.pop("urgent_fifo", a.urgent_fifo)
             kw.update(miss_correction=True, urgent_stream=self.copy if fifo else self.torch.cuda.Stream(priority=-1))

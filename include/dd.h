@@ -56,6 +56,7 @@ extern "C" {
 #define DD_ATTN_AUTO    0           /* the faster one as measured: the split-KV kernel */
 #define DD_ATTN_SPLIT   1           /* split-KV kernel: grid (split, KV head, request), cluster merge */
 #define DD_ATTN_STREAM  2           /* streaming kernel: equal runs of pages per block, TMA-fed shared-memory ring */
+#define DD_ATTN_TC      3           /* the streaming split on tcgen05: tiles of 8 pages, accumulators in tensor memory */
 
 #define DD_SELECT_AUTO         0    /* fused cluster kernel when the request fits, else the two-kernel path */
 #define DD_SELECT_TWO_KERNELS  1    /* scoring kernel + top-k kernel with logits in global scratch */
@@ -91,7 +92,7 @@ typedef struct dd_config {
                                 copy engine, shorter ones through the zero-copy kernel; 0 = library default (8) */
   int stage_block_pages;     /* DD_GATHER_STAGED: 0 = copy exactly the selected runs; 2, 4, 8, 16 or 32 = copy every
                                 aligned block of that many pages that holds a selected page (over-fetch, no stragglers) */
-  int attn_mode;             /* DD_ATTN_AUTO, DD_ATTN_SPLIT or DD_ATTN_STREAM (attn_splits applies to the split kernel) */
+  int attn_mode;             /* DD_ATTN_AUTO, DD_ATTN_SPLIT, DD_ATTN_STREAM or DD_ATTN_TC (attn_splits applies to the split kernel) */
 } dd_config;
 
 /* ---- context ------------------------------------------------------------------------------- */

@@ -32,6 +32,7 @@ DD_TRACE_FIELDS = 8
 DD_ATTN_AUTO = 0
 DD_ATTN_SPLIT = 1
 DD_ATTN_STREAM = 2
+DD_ATTN_TC = 3
 DD_SELECT_AUTO = 0
 DD_SELECT_TWO_KERNELS = 1
 

@@ -70,7 +70,9 @@ static const char* dd_check_config(const dd_config* c) {
     const int ct = c->landmark_chunk_tokens;
     if (ct != 0 && ct != 16 && ct != 8 && ct != 4 && ct != 2 && ct != 1) return "landmark_chunk_tokens must be 0, 16, 8, 4, 2 or 1";
   }
-  if (c->attn_mode != DD_ATTN_AUTO && c->attn_mode != DD_ATTN_SPLIT && c->attn_mode != DD_ATTN_STREAM) return "unknown attn_mode";
+  if (c->attn_mode != DD_ATTN_AUTO && c->attn_mode != DD_ATTN_SPLIT && c->attn_mode != DD_ATTN_STREAM &&
+      c->attn_mode != DD_ATTN_TC)
+    return "unknown attn_mode";
   if (c->attn_splits > 512) return "attn_splits must be <= 512";
   if (c->attn_splits > 64 && c->attn_splits % 8) return "attn_splits above 64 must be a multiple of 8";
   if ((long long)c->batch * c->n_kv_heads * c->k_pages > 0x7fffffffLL) return "too many selected pages";
@@ -127,8 +129,10 @@ static dd_sizes dd_compute_sizes(const dd_config* c, int S, int sm_count) {
   z.topk_keys = up256(B * Hkv * P * 4);
   {
     // partials of the split-KV kernel (S per unit) or of the streaming kernel (max_parts per unit), whichever is larger
-    int nb = 0, ppb = 0, parts = 0;
+    int nb = 0, ppb = 0, parts = 0, parts_tc = 0;
     dd_attn_stream_geometry(c, sm_count, &nb, &ppb, &parts);
+    dd_attn_tc_geometry(c, sm_count, &nb, &ppb, &parts_tc);
+    if (parts_tc > parts) parts = parts_tc;
     const size_t n_part = (size_t)(S > parts ? S : parts);
     z.part_o = up256(B * Hkv * n_part * 8 * DD_D * 4);
     z.part_ml = up256(B * Hkv * n_part * 8 * 8);
@@ -334,8 +338,9 @@ extern "C" int dd_create(const dd_config* cfg, dd_ctx** out) {
   }
   int rc = dd_select_setup(ctx);
   if (rc == DD_OK) rc = dd_gather_setup(ctx);
-  ctx->attn_stream = cfg->attn_mode == DD_ATTN_STREAM;   // measured slower than the split-KV kernel: opt-in only
-  if (rc == DD_OK && ctx->attn_stream) rc = dd_attn_stream_setup(ctx);
+  ctx->attn_stream = cfg->attn_mode == DD_ATTN_STREAM ? 1 : (cfg->attn_mode == DD_ATTN_TC ? 2 : 0);   // both opt-in
+  if (rc == DD_OK && ctx->attn_stream == 1) rc = dd_attn_stream_setup(ctx);
+  if (rc == DD_OK && ctx->attn_stream == 2) rc = dd_attn_tc_setup(ctx);
   if (rc == DD_OK && ctx->attn_stream && cudaEventCreate(&ctx->as_fence) != cudaSuccess) {
     snprintf(ctx->errmsg, sizeof(ctx->errmsg), "dd_create: cannot create the streaming kernel's fence event");
     rc = DD_ERR_CUDA;

@@ -447,7 +447,10 @@ static cudaError_t dd_attn_launch_raw(cudaStream_t st, int batch, int Hkv, int G
 int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx, const int* ctx_len, void* out,
                    float* out_lse, cudaStream_t st, const void* k_new, const void* v_new) {
   const dd_config& c = ctx->cfg;
-  if (ctx->attn_stream)       // every slot of the ring has its tensor map
+  if (ctx->attn_stream == 2)  // every slot of the ring has its tensor maps
+    return dd_launch_attn_tc(ctx, q, (int)((size_t)(slot - ctx->ring) / ctx->slot_bytes), idx, ctx_len, out, out_lse, st,
+                             k_new, v_new);
+  if (ctx->attn_stream)
     return dd_launch_attn_stream(ctx, q, (int)((size_t)(slot - ctx->ring) / ctx->slot_bytes), idx, ctx_len, out, out_lse, st,
                                  k_new, v_new, false);
   DD_CUDA_TRY(ctx, dd_attn_launch_raw(st, c.batch, c.n_kv_heads, ctx->G, c.n_q_tokens, c.k_pages, ctx->attn_splits,
@@ -488,7 +491,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 4) dd_attn_loads_only_kernel(con
 
 int dd_launch_attn_loads_only(dd_ctx* ctx, const char* slot, cudaStream_t st) {
   const dd_config& c = ctx->cfg;
-  if (ctx->attn_stream)
+  if (ctx->attn_stream == 1)
     return dd_launch_attn_stream(ctx, nullptr, (int)((size_t)(slot - ctx->ring) / ctx->slot_bytes), nullptr, nullptr, nullptr,
                                  nullptr, st, nullptr, nullptr, true);
   const int S = ctx->attn_splits;

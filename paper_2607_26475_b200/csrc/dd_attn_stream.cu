@@ -483,9 +483,9 @@ typedef CUresult (*dd_encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint
                                        const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// Tensor map of one ring slot seen as [rows = B * Hkv * 2 * k * T][128 channels] bf16, boxes of 16 rows x 64 channels
+// Tensor map of one ring slot seen as [rows = B * Hkv * 2 * k * T][128 channels] bf16, boxes of box_rows rows x 64 channels
 // with the 128-byte swizzle. Returns DD_OK, or an error when the driver entry point is missing or refuses the map.
-int dd_attn_stream_make_map(dd_ctx* ctx, const void* slot, void* map_out) {
+int dd_attn_stream_make_map(dd_ctx* ctx, const void* slot, void* map_out, int box_rows) {
   static dd_encode_tiled_fn encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -500,7 +500,7 @@ int dd_attn_stream_make_map(dd_ctx* ctx, const void* slot, void* map_out) {
   const dd_config& c = ctx->cfg;
   const cuuint64_t dims[2] = {(cuuint64_t)DD_D, (cuuint64_t)c.batch * c.n_kv_heads * 2 * c.k_pages * DD_T};
   const cuuint64_t strides[1] = {(cuuint64_t)DD_ROW_BYTES};
-  const cuuint32_t box[2] = {64, (cuuint32_t)DD_T};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t elem[2] = {1, 1};
   const CUresult r = encode((CUtensorMap*)map_out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(slot), dims, strides,
                             box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -514,7 +514,7 @@ int dd_attn_stream_setup(dd_ctx* ctx) {
   DD_CUDA_TRY(ctx, cudaFuncSetAttribute(dd_attn_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AS_SMEM_BYTES));
   dd_attn_stream_geometry(&ctx->cfg, ctx->sm_count, &ctx->as_blocks, &ctx->as_ppb, &ctx->as_max_parts);
   for (int s = 0; s < ctx->cfg.ring_depth; ++s) {
-    const int rc = dd_attn_stream_make_map(ctx, ctx->ring + (size_t)s * ctx->slot_bytes, &ctx->as_tmap[s]);
+    const int rc = dd_attn_stream_make_map(ctx, ctx->ring + (size_t)s * ctx->slot_bytes, &ctx->as_tmap[s], DD_T);
     if (rc != DD_OK) return rc;
   }
   return DD_OK;

@@ -28,10 +28,11 @@ struct dd_ctx {
   int score_tiles;       // ceil(P / DD_SCORE_TILE)
   int attn_splits;       // resolved blocks per (request, KV head)
   int attn_cluster;      // blocks per thread-block cluster (divides attn_splits)
-  int attn_stream;       // 1: the streaming attention kernel serves the context's calls, 0: the split-KV kernel
+  int attn_stream;       // which attention kernel serves the context's calls: 0 split-KV, 1 streaming, 2 tcgen05
   cudaEvent_t as_fence;  // timing-enabled event recorded behind the streaming kernel inside the layer step (see dd_api.cu)
   int as_blocks, as_ppb, as_max_parts;   // streaming kernel: grid, pages per block, partials per unit
-  struct alignas(64) { unsigned char bytes[128]; } as_tmap[DD_MAX_RING];   // tensor map of every ring slot
+  struct alignas(64) { unsigned char bytes[128]; } as_tmap[DD_MAX_RING];   // tensor map of every ring slot, page boxes
+  struct alignas(64) { unsigned char bytes[128]; } tc_tmap[DD_MAX_RING];   // the same with boxes of a tile (128 rows)
   int sel_cluster;       // blocks per cluster of the fused selection kernel; 0 = two-kernel path
   int sel_ppc;           // pages per block of the fused selection
   int sel_smem_bytes;
@@ -140,6 +141,11 @@ int dd_launch_attn(dd_ctx* ctx, const void* q, const char* slot, const int* idx,
 int dd_launch_attn_loads_only(dd_ctx* ctx, const char* slot, cudaStream_t st);
 void dd_attn_stream_geometry(const dd_config* c, int sm_count, int* n_blocks, int* ppb, int* max_parts);
 int dd_attn_stream_setup(dd_ctx* ctx);
+int dd_attn_stream_make_map(dd_ctx* ctx, const void* slot, void* map_out, int box_rows);
+void dd_attn_tc_geometry(const dd_config* c, int sm_count, int* n_blocks, int* ppb, int* max_parts);
+int dd_attn_tc_setup(dd_ctx* ctx);
+int dd_launch_attn_tc(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len, void* out, float* out_lse,
+                      cudaStream_t st, const void* k_new, const void* v_new);
 int dd_launch_attn_stream(dd_ctx* ctx, const void* q, int slot, const int* idx, const int* ctx_len, void* out,
                           float* out_lse, cudaStream_t st, const void* k_new, const void* v_new, bool probe);
 int dd_launch_select_loads_only(dd_ctx* ctx, const void* landmarks, const int* n_pages, cudaStream_t st);

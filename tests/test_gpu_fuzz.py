@@ -55,8 +55,8 @@ def _attn_shapes(n, seed):
 
 
 @pytest.mark.parametrize("seed", [1, 2, 3])
-@pytest.mark.parametrize("mode", ["split", "stream"])
+@pytest.mark.parametrize("mode", ["split", "stream", "tc"])
 def test_attention_on_random_shapes(dd, seed, mode):
-    attn_mode = dd.DD_ATTN_STREAM if mode == "stream" else dd.DD_ATTN_SPLIT
+    attn_mode = {"stream": dd.DD_ATTN_STREAM, "split": dd.DD_ATTN_SPLIT, "tc": dd.DD_ATTN_TC}[mode]
     for B, P, k, ctx_len, Tq, splits, s, G in _attn_shapes(6, seed):
         _attn_case(dd, B, P, k, ctx_len, Tq, splits, seed=s, G=G, attn_mode=attn_mode)

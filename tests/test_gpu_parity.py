@@ -23,10 +23,10 @@ def dd():
     return binding
 
 
-@pytest.fixture(params=["stream", "split"])
+@pytest.fixture(params=["stream", "split", "tc"])
 def attn_mode(request, dd):
-    """Both attention kernels serve the same entry points."""
-    return dd.DD_ATTN_STREAM if request.param == "stream" else dd.DD_ATTN_SPLIT
+    """All three attention kernels serve the same entry points."""
+    return {"stream": dd.DD_ATTN_STREAM, "split": dd.DD_ATTN_SPLIT, "tc": dd.DD_ATTN_TC}[request.param]
 
 
 def _layer_store(w, layer, pinned=True):
@@ -256,11 +256,13 @@ def test_attention_sharp_queries_and_other_group_sizes(dd, attn_mode):
     _attn_case(dd, 1, 128, 32, [2048], 2, 2, seed=4, G=1, attn_mode=attn_mode)
 
 
-def test_streaming_attention_when_blocks_cut_units_at_every_offset(dd):
+@pytest.mark.parametrize("mode", ["stream", "tc"])
+def test_streaming_attention_when_blocks_cut_units_at_every_offset(dd, mode):
     """Shapes whose flat page list is cut into per-block runs that start and end inside units, cover several whole
-    units, or hold fewer pages than consumer warps: many requests with few pages, one request with many."""
+    units, or hold fewer pages than consumer warps (or than a tile): many requests with few pages, one with many."""
+    attn_mode = dd.DD_ATTN_STREAM if mode == "stream" else dd.DD_ATTN_TC
     for B, P, k, seed in [(16, 40, 5, 1), (9, 64, 7, 2), (1, 4096, 1200, 3), (5, 200, 66, 4), (32, 64, 64, 5)]:
-        _attn_case(dd, B, P, k, [P * 16 - (3 * b) % 15 for b in range(B)], 2, 0, seed=seed, attn_mode=dd.DD_ATTN_STREAM)
+        _attn_case(dd, B, P, k, [P * 16 - (3 * b) % 15 for b in range(B)], 2, 0, seed=seed, attn_mode=attn_mode)
 
 
 def test_full_budget_equals_dense_attention(dd):

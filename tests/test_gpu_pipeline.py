@@ -95,16 +95,19 @@ def test_chain_matches_oracle_and_is_invariant_to_ring_depth_and_engine(dd):
             assert np.array_equal(i2, idxs)
 
 
-def test_chain_with_the_streaming_attention_kernel(dd):
-    """The pipelined step with the TMA-fed attention kernel: same index sets, outputs equal to the split-KV
-    kernel's up to rounding (the two merge partial results in different orders) and within tolerance of the oracle."""
+@pytest.mark.parametrize("mode", ["stream", "tc"])
+def test_chain_with_the_streaming_attention_kernel(dd, mode):
+    """The pipelined step with the TMA-fed attention kernels (mma.sync consumers, or tcgen05 with accumulators in tensor
+    memory): same index sets, outputs equal to the split-KV kernel's up to rounding (partial results are merged in
+    different orders) and within tolerance of the oracle."""
+    attn_mode = dd.DD_ATTN_STREAM if mode == "stream" else dd.DD_ATTN_TC
     S = 3
     w = wl.small(wl.CONFIGS[4], n_layers=3, batch=2, ctx=16 * 90, budget=16 * 12, recent_window=32)
     inp = _inputs(w, S)
     store, lms, ctx_len, npg, q_init, q_steps = inp
     want, want_idx = _run(dd, w, S, inp, depth=2)
     for depth in (2, 3):
-        got, got_idx = _run(dd, w, S, inp, depth=depth, ctx_kw=dict(attn_mode=dd.DD_ATTN_STREAM))
+        got, got_idx = _run(dd, w, S, inp, depth=depth, ctx_kw=dict(attn_mode=attn_mode))
         assert np.array_equal(got_idx, want_idx)
         assert np.abs(f32(got) - f32(want)).max() <= 2e-2
         for t in range(S):
