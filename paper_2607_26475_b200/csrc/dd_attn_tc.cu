@@ -5,12 +5,14 @@
 // block the pages of a unit are taken in tiles of eight (128 tokens):
 //   warp 4, one thread   TMA: the tile's K and V rows into a three-deep shared-memory ring, 128-byte swizzle, one
 //                        [64 channels x 128 rows] box per (K | V, channel half); partial tiles page by page
-//   warp 5, one thread   tcgen05.mma, accumulators in tensor memory:
+//   warps 5 and 6, one   tcgen05.mma, accumulators in tensor memory (an issuing thread per product: issuing costs
+//   thread each          40-70 ns per instruction whatever its size, the tensor pipe itself is busy 2% of the time):
 //                          S^T[128 tokens x 16] = K[128 x 128] . q^T          (A = K tile, K-major; B = q, rows 8..15 zero)
 //                          O^T[128 channels x 16] += V^T[128 x 16 tokens] . P^T   per page (A = V, MN-major; B = P)
 //   warps 0-3            one thread per token of the tile: S from tensor memory, running soft-max over tiles, P
-//                        (bf16) into shared memory as the next B operand; O is rescaled in tensor memory only when
-//                        a row's reference maximum moves; at the end of a unit's pages thread d owns channel d of O
+//                        (bf16) into shared memory as the next B operand; S and P are double-buffered, O is rescaled
+//                        in tensor memory only when a row's reference maximum moves by more than 2^8; at the end of a
+//                        unit's pages thread d owns channel d of O
 // The up-to-8 query rows of a KV head are the N columns (padded to 16, the smallest N for M = 128). All waits on
 // mbarriers are bounded; a wait that gives up sets the device error word and the block runs out without waiting
 // again, frees its tensor memory and returns.
@@ -19,7 +21,7 @@
 #include "dd_common.cuh"
 
 constexpr int TC_EPI = 4;                              // soft-max / epilogue warps = 128 tensor-memory lanes
-constexpr int TC_THREADS = (TC_EPI + 2) * 32;
+constexpr int TC_THREADS = (TC_EPI + 3) * 32;           // + TMA warp, S^T issuer, O^T issuer
 constexpr int TC_TILE_PAGES = 8;
 constexpr int TC_TILE_TOKENS = TC_TILE_PAGES * DD_T;   // 128
 constexpr int TC_HALF_BYTES = TC_TILE_TOKENS * 128;    // one (K | V, channel half) of a tile: 128 rows of 128 B
@@ -279,17 +281,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) dd_attn_tc_kernel(
     }
     __syncwarp();
   } else if (warp == TC_EPI + 1) {
-    // ---- one thread issues the matrix products
+    // ---- one thread issues S^T = K q^T. Issuing costs 40-70 ns per tcgen05.mma whatever its size (measured), so the
+    // two products have an issuing thread each. S^T of tile t goes to buffer t % 2 as soon as the soft-max of tile
+    // t - 2 has read it, also across a unit boundary (the q operand of unit s sits in buffer s % 2, written a unit ahead).
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = tc_idesc(128, TC_N, 0);
-      constexpr uint32_t IDESC_PV = tc_idesc(128, TC_N, 1);
-      const uint32_t tmem_o = tmem_base + 2 * TC_N;
-      // S^T of tile t goes to buffer t % 2: it is issued while the soft-max of tile t - 1 is still at work, also across
-      // a unit boundary (the q operand of unit s sits in buffer s % 2 and is written one unit ahead)
-      auto issue_qk = [&](const tc_iter& it) -> bool {
-        if (it.first() && !tc_wait(tc_smem(&q_bar[it.seg_no & 1]), (uint32_t)((it.seg_no >> 1) & 1), abort_p, wait_ns)) return false;
+      tc_iter it;
+      for (it.start(f0, f1, k); it.valid(); it.next()) {
         const int t = it.tile_no, s = t % TC_STAGES, round = t / TC_STAGES;
-        if (!tc_wait(tc_smem(&full_bar[s]), (uint32_t)(round & 1), abort_p, wait_ns)) return false;
+        if (it.first() && !tc_wait(tc_smem(&q_bar[it.seg_no & 1]), (uint32_t)((it.seg_no >> 1) & 1), abort_p, wait_ns)) break;
+        if (t >= 2 && !tc_wait(tc_smem(&p_ready_bar[t & 1]), (uint32_t)(((t - 2) >> 1) & 1), abort_p, wait_ns)) break;
+        if (!tc_wait(tc_smem(&full_bar[s]), (uint32_t)(round & 1), abort_p, wait_ns)) break;
         tc_fence_after();
         const uint32_t stage = ring + (uint32_t)s * TC_TILE_BYTES;
         const uint32_t qb = q_smem + (it.seg_no & 1) * TC_B_BYTES;
@@ -300,19 +302,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) dd_attn_tc_kernel(
           tc_mma(tmem_base + (t & 1) * TC_N, a, bq, IDESC_QK, kk > 0 ? 1u : 0u);
         }
         tc_commit(tc_smem(&s_full_bar[t & 1]));
-        return true;
-      };
+      }
+    }
+    __syncwarp();
+  } else if (warp == TC_EPI + 2) {
+    // ---- one thread issues O^T += V^T P^T, page by page, and releases the tile's ring stage (its S^T product was
+    // complete before the soft-max that produced this P could start)
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = tc_idesc(128, TC_N, 1);
+      const uint32_t tmem_o = tmem_base + 2 * TC_N;
       tc_iter it;
-      it.start(f0, f1, k);
-      bool ok = it.valid() && issue_qk(it);
-      while (ok && it.valid()) {
-        tc_iter nx = it;
-        nx.next();
-        if (nx.valid() && !issue_qk(nx)) break;
-        const int t = it.tile_no, np = it.np();
+      for (it.start(f0, f1, k); it.valid(); it.next()) {
+        const int t = it.tile_no, s = t % TC_STAGES, round = t / TC_STAGES, np = it.np();
+        if (!tc_wait(tc_smem(&full_bar[s]), (uint32_t)(round & 1), abort_p, wait_ns)) break;
         if (!tc_wait(tc_smem(&p_ready_bar[t & 1]), (uint32_t)((t >> 1) & 1), abort_p, wait_ns)) break;
         tc_fence_after();
-        const uint32_t stage = ring + (uint32_t)(t % TC_STAGES) * TC_TILE_BYTES;
+        const uint32_t stage = ring + (uint32_t)s * TC_TILE_BYTES;
 #pragma unroll
         for (int p = 0; p < TC_TILE_PAGES; ++p) {
           if (p >= np) break;
@@ -320,9 +325,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) dd_attn_tc_kernel(
           const uint64_t bp = tc_desc(p_smem + (t & 1) * TC_B_BYTES + p * 512, 256, 128, 0);
           tc_mma(tmem_o, a, bp, IDESC_PV, (it.first() && p == 0) ? 0u : 1u);
         }
-        tc_commit(tc_smem(&empty_bar[t % TC_STAGES]));
+        tc_commit(tc_smem(&empty_bar[s]));
         tc_commit(tc_smem(&pv_done_bar[t & 1]));
-        it = nx;
       }
     }
     __syncwarp();
