@@ -98,6 +98,13 @@ int dd_test_pick_cluster(int max_pages, int problems, int sm_count, int rows_per
                          int (*fits)(int blocks, size_t shared_bytes, void* user), void* user, int* pages_per_block,
                          size_t* shared_bytes, int* ring_stages, int* logits_global);
 
+/* Test hook, needs no GPU: the flat work split of the two TMA-fed attention kernels (kind 0: streaming kernel, two
+ * blocks per SM; kind 1: tcgen05 kernel, one block per SM) for a launch of batch * n_kv_heads units of k_pages pages.
+ * Block x owns the pages [x * pages_per_block, (x + 1) * pages_per_block) of the flat list; max_parts is the number of
+ * partial results reserved per unit. Returns DD_OK or DD_ERR_INVALID_ARG. */
+int dd_test_attn_split(int kind, int batch, int n_kv_heads, int k_pages, int sm_count, int* n_blocks, int* pages_per_block,
+                       int* max_parts);
+
 #ifdef __cplusplus
 }
 #endif

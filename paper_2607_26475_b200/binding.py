@@ -44,7 +44,7 @@ EXPORTS = [
     "dd_select_topk_chunked", "dd_sparse_decode_attn_causal", "dd_decode_layer_step_causal", "dd_diff_indices",
     "dd_fetch_missing_from_host", "dd_get_merged_indices", "dd_miss_stats", "dd_probe_attn_loads", "dd_probe_select_loads",
     "dd_trace_begin", "dd_trace_end", "dd_trace_read", "dd_decode_step_host", "dd_last_device_error",
-    "dd_gather_stats", "dd_set_bulk_wait", "dd_test_pick_cluster", "dd_test_stage_plan",
+    "dd_gather_stats", "dd_set_bulk_wait", "dd_test_pick_cluster", "dd_test_stage_plan", "dd_test_attn_split",
 ]
 
 
@@ -119,6 +119,7 @@ def _load() -> C.CDLL:
     lib.dd_set_bulk_wait.argtypes = [vp, C.c_double, ip]
     lib.dd_test_pick_cluster.argtypes = [ip, ip, ip, ip, ip, ip, PICK_FITS, vp, C.POINTER(ip), C.POINTER(C.c_size_t), C.POINTER(ip), C.POINTER(ip)]
     lib.dd_test_stage_plan.argtypes = [vp, vp, ip, ip, ip, ip, ip, ip, C.c_longlong, vp, C.c_longlong, vp, vp, vp, vp, vp, vp]
+    lib.dd_test_attn_split.argtypes = [ip, ip, ip, ip, ip, C.POINTER(ip), C.POINTER(ip), C.POINTER(ip)]
     lib.dd_static_scratch_capacity.argtypes = []
     lib.dd_static_scratch_capacity.restype = C.c_size_t
     lib.dd_sparse_decode_attn_static.argtypes = [ip] * 8 + [vp] * 7

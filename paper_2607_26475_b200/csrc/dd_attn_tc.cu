@@ -666,3 +666,15 @@ int dd_launch_attn_tc(dd_ctx* ctx, const void* q, int slot, const int* idx, cons
                                       ctx->err_word, ctx->bulk_wait_ns));
   return DD_OK;
 }
+
+extern "C" int dd_test_attn_split(int kind, int batch, int n_kv_heads, int k_pages, int sm_count, int* n_blocks,
+                                  int* pages_per_block, int* max_parts) {
+  if ((kind != 0 && kind != 1) || batch < 1 || n_kv_heads < 1 || k_pages < 1 || sm_count < 1 || !n_blocks || !pages_per_block ||
+      !max_parts)
+    return DD_ERR_INVALID_ARG;
+  dd_config c = {};
+  c.batch = batch; c.n_kv_heads = n_kv_heads; c.k_pages = k_pages;
+  if (kind == 0) dd_attn_stream_geometry(&c, sm_count, n_blocks, pages_per_block, max_parts);
+  else dd_attn_tc_geometry(&c, sm_count, n_blocks, pages_per_block, max_parts);
+  return DD_OK;
+}

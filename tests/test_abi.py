@@ -87,3 +87,27 @@ def test_cluster_search_of_the_fused_selection_always_terminates():
     # a larger cluster is used when the preferred one cannot hold all its clusters
     got, calls = pick(2048, 64, 1, 1, lambda c, s: 64 if c >= 8 else 10)
     assert got == 8 and [c for c, _ in calls] == [4, 8]
+
+
+def test_flat_work_split_of_the_tma_fed_attention_kernels():
+    """Block x owns pages [x * ppb, (x + 1) * ppb) of the flat list of B * Hkv * k pages: the blocks cover the list, no
+    unit is cut into more parts than reserved for it (at most 64), and large launches use every SM."""
+    import ctypes
+    from paper_2607_26475_b200 import binding
+    rng = __import__("random").Random(3)
+    shapes = [(8, 8, 128), (32, 8, 64), (8, 8, 256), (1, 8, 512), (1, 8, 16), (1, 1, 1), (1, 8, 8192), (64, 8, 3), (5, 8, 66)]
+    shapes += [(rng.randint(1, 40), rng.choice([1, 2, 8]), rng.randint(1, 3000)) for _ in range(200)]
+    for kind, per_sm, min_pages in ((0, 2, 8), (1, 1, 8)):
+        for B, Hkv, k in shapes:
+            nb, ppb, parts = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+            assert binding.lib.dd_test_attn_split(kind, B, Hkv, k, 148, ctypes.byref(nb), ctypes.byref(ppb), ctypes.byref(parts)) == 0
+            nb, ppb, parts = nb.value, ppb.value, parts.value
+            total = B * Hkv * k
+            assert nb >= 1 and ppb >= 1 and (nb - 1) * ppb < total <= nb * ppb          # covers the list, no empty block
+            assert nb <= per_sm * 148
+            worst = max(((u + 1) * k - 1) // ppb - (u * k) // ppb + 1 for u in range(min(B * Hkv, 400)))
+            assert worst <= parts <= 64
+            ppb_free = -(-total // (per_sm * 148))                                      # without the limit on parts per unit
+            if total >= per_sm * 148 * min_pages and (k - 1) // ppb_free + 2 <= 64:
+                assert nb >= per_sm * 148 - per_sm * 148 // 8                          # a large launch keeps the SMs busy
+    assert binding.lib.dd_test_attn_split(2, 1, 1, 1, 148, None, None, None) != 0
